@@ -1,0 +1,147 @@
+/*
+ * mpq -- multi-precision quantized layers through the {-1,+1} encoding decomposition,
+ * for NVIDIA B200 (sm_100a).  C ABI of libmpq.so.
+ *
+ * The method (Sun et al., "Multi-Precision Quantized Neural Networks via Encoding
+ * Decomposition of {-1,+1}"): an activation of a_bits and a weight of w_bits are
+ * quantized to odd integers, written as sum_p 2^p c_p with c_p in {-1,+1} (Eq. 10),
+ * stored one bit per element in bit-planes, and every dot product of a layer becomes
+ * a_bits x w_bits binary-branch dot products (Eq. 7-9), each computed with xor and
+ * bitcount, weighted 2^(i+j), summed, and scaled back to a real number (Eq. 18).
+ *
+ * Conventions for every entry point
+ *   - Pointers are DEVICE pointers unless the name ends in _host.  The caller owns and
+ *     sizes every buffer; the library allocates nothing and keeps no state between calls
+ *     (exception: mpq_linear_host stages through a caller-provided device workspace).
+ *   - Calls are asynchronous on `stream` (a cudaStream_t passed as void*; NULL = the
+ *     default stream) unless stated otherwise.  Outputs are fully overwritten.
+ *   - Return value: an mpq_status.  Errors that the host can see (null pointers, bad
+ *     sizes, unsupported widths, int32 headroom) are returned before anything is
+ *     launched; a launch failure maps to MPQ_ERR_CUDA.  Nothing aborts or traps.
+ *   - Bit-widths are 1..8 for both operands (the paper's 64 encoding choices, Section 5.1).
+ *
+ * Packed layout ("planes")
+ *   planes[p][row][word], p = 0..bits-1, word = 0..mpq_row_words(k)-1, uint32.
+ *   Bit t of word w of a row is element 32*w + t of that row.  Bit value 1 is +1, 0 is -1.
+ *   Plane p holds bit p of the level index u = (q + 2^bits - 1)/2 and carries weight 2^p
+ *   (plane 0 is the low bit: "x = x1 + 2 x2").  Bits past element k-1 and the words that
+ *   pad a row to a multiple of 4 words are 0 in every operand.
+ */
+#ifndef MPQ_H_
+#define MPQ_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    MPQ_OK = 0,
+    MPQ_ERR_NULL = 1,        /* a required pointer is NULL                                   */
+    MPQ_ERR_BAD_SHAPE = 2,   /* a size is negative/zero where it may not be, or ld < extent  */
+    MPQ_ERR_UNSUPPORTED = 3, /* bits outside 1..8; kernel not 1x1/3x3; stride not 1/2;
+                                pad > 1; C not 32, 64 or a multiple of 128; unknown enum     */
+    MPQ_ERR_OVERFLOW = 4,    /* k * (2^a_bits-1) * (2^w_bits-1) >= 2^31: int32 would overflow */
+    MPQ_ERR_ALIGN = 5,       /* a plane pointer is not 16-byte aligned                       */
+    MPQ_ERR_CUDA = 6,        /* the CUDA runtime reported an error (launch, copy)            */
+    MPQ_ERR_WORKSPACE = 7    /* caller-provided workspace is too small                       */
+} mpq_status;
+
+typedef enum { MPQ_SCALE_PER_TENSOR = 0, MPQ_SCALE_PER_ROW = 1 } mpq_scale_mode;
+
+/* Range limiter applied before the quantizer (Table 1): HTanh clamps x/s to [-1,1],
+ * HReLU clamps it to [0,1] (negative inputs land on the level just above zero). */
+typedef enum { MPQ_ACT_HTANH = 0, MPQ_ACT_HRELU = 1 } mpq_act;
+
+const char* mpq_status_string(int status);
+
+/* Words per packed row: ceil(k/32) rounded up to a multiple of 4 (rows are 16-byte multiples).
+ * Storage is bits/32 of the fp32 tensor plus this padding (the paper's memory saving). */
+int64_t mpq_row_words(int64_t k);
+/* Words of a whole packed operand: bits * rows * mpq_row_words(k).  0 on invalid arguments. */
+int64_t mpq_packed_words(int64_t rows, int64_t k, int bits);
+
+/* ---- Range.  BASELINE generalisation of the paper's fixed [-1,1] / [0,1] ranges (Table 1):
+ * scale_out = max |x| (HTanh) or max of max(x,0) (HReLU), NaNs ignored; one value
+ * (PER_TENSOR) or one per row (PER_ROW).  x is [rows x k] with row stride ldx (elements).
+ * scale_out is overwritten (the call zeroes it first, on the stream). */
+int mpq_absmax(const float* x, int64_t rows, int64_t k, int64_t ldx, int mode, int act,
+               float* scale_out, void* stream);
+
+/* ---- Encoder (Fig. 1 "Encoder"; quantizer Eq. 15 with round-half-up; code Table 2 / Eq. 10;
+ * one bit per element, Section 1 "store by bit vectors").
+ * Per element, in fp32: inv = 1/s (0 if s is not a finite positive number),
+ * y = (x*inv) * ((2^bits-1)/2) as two rounded multiplies, NaN -> 0, HReLU: max(y,0),
+ * clamp to [-2^(bits-1), 2^(bits-1)-1/2], u = floor(y) + 2^(bits-1).  Plane p gets bit p of u.
+ * x: [rows x k], row stride ldx; scale: 1 value or `rows` values; planes: mpq_packed_words(). */
+int mpq_encode(const float* x, int64_t rows, int64_t k, int64_t ldx,
+               const float* scale, int mode, int act, int bits,
+               uint32_t* planes, void* stream);
+
+/* Activations for mpq_conv: x [N][C][H][W] fp32 -> planes[bits][N][H][W][C/32]
+ * (channel innermost: bit t of word cw at a pixel is channel 32*cw + t).  One range value.
+ * C must be 32, 64 or a multiple of 128. */
+int mpq_encode_nchw(const float* x, int N, int C, int H, int W, const float* scale, int act,
+                    int bits, uint32_t* planes, void* stream);
+
+/* Weights for mpq_conv: w [O][C][KH][KW] fp32 -> planes[bits][O][mpq_row_words(KH*KW*C)], the
+ * row of output channel o ordered (kh, kw, c) with c innermost.  scale: 1 value or O values.
+ * tap_sums [KH*KW][O] int32 (required): sum over c of the decoded weight q_w[o][c][kh][kw];
+ * mpq_conv uses it to make out-of-image taps contribute exactly 0. */
+int mpq_encode_oihw(const float* w, int O, int C, int KH, int KW, const float* scale, int mode,
+                    int bits, uint32_t* planes, int32_t* tap_sums, void* stream);
+
+/* ---- Layer product (Eq. 7-10 branches, xor + bitcount; Fig. 1 "Decoder"; scale Eq. 18).
+ * C = A * B^T with A = a_planes [a_bits][m][rw], B = b_planes [b_bits][n][rw], rw = mpq_row_words(k):
+ *   S        = sum_{i<a_bits, j<b_bits} 2^(i+j) * sum_w popcount(A_i[r][w] xor B_j[c][w])
+ *   c_i32    = (2^a_bits-1)(2^b_bits-1) k - 2 S           (= sum_t q_a[r][t] q_b[c][t], exact)
+ *   c_f32    = float(c_i32) * ((a_scale/(2^a_bits-1)) * (b_scale[c]/(2^b_bits-1)))
+ * c_i32 and c_f32 are [m x n] row-major with row stride ldc; either may be NULL, not both.
+ * a_scale: 1 value; b_scale: 1 value (PER_TENSOR) or n values (PER_ROW); both may be NULL
+ * when c_f32 is NULL.  No bias ("we suppose the bias does not exist"). */
+int mpq_gemm(const uint32_t* a_planes, int a_bits, const uint32_t* b_planes, int b_bits,
+             int64_t m, int64_t n, int64_t k,
+             int32_t* c_i32, float* c_f32, int64_t ldc,
+             const float* a_scale, const float* b_scale, int b_mode, void* stream);
+
+/* ---- Convolution by the same decomposition ("convolution ... layers are also suit"),
+ * done as an implicit im2col on the packed planes: GEMM row = output pixel (n, oh, ow),
+ * GEMM k = (kh, kw, c).  x_planes from mpq_encode_nchw, w_planes and tap_sums from
+ * mpq_encode_oihw.  3x3 or 1x1, stride 1 or 2, pad 0 or 1, true zero padding (a tap outside
+ * the image adds 0 to the integer sum).  y [N][O][Ho][Wo], Ho = (H + 2 pad - KH)/stride + 1.
+ * y_i32 / y_f32: either may be NULL, not both.  w_scale: 1 or O values. */
+int mpq_conv(const uint32_t* x_planes, int a_bits, int N, int C, int H, int W,
+             const uint32_t* w_planes, int w_bits, const int32_t* tap_sums,
+             int O, int KH, int KW, int stride, int pad,
+             int32_t* y_i32, float* y_f32,
+             const float* x_scale, const float* w_scale, int w_mode, void* stream);
+
+/* ---- Glue for chained layers (not part of the paper's method): y = max(a + b, 0) elementwise,
+ * b may be NULL (plain ReLU).  n elements, fp32, one rounded add. */
+int mpq_add_relu(const float* a, const float* b, float* y, int64_t n, void* stream);
+
+/* ---- Whole encoded fully-connected layer from HOST buffers (Fig. 1 end to end):
+ * copies x_host [m x k] and w_host [n x k] to the device workspace, takes both ranges
+ * (activations per tensor with `a_act`, weights per `w_mode`), encodes both, runs mpq_gemm,
+ * and copies out_i32_host / out_f32_host [m x n] back (either may be NULL, not both).
+ * Host buffers should be pinned for the copies to be asynchronous.  The call returns after
+ * the stream has drained (it synchronizes `stream`).
+ * workspace: device memory of at least mpq_linear_host_workspace() bytes, 256-byte aligned. */
+int64_t mpq_linear_host_workspace(int64_t m, int64_t n, int64_t k, int a_bits, int w_bits);
+int mpq_linear_host(const float* x_host, const float* w_host, int64_t m, int64_t n, int64_t k,
+                    int a_bits, int w_bits, int a_act, int w_mode,
+                    int32_t* out_i32_host, float* out_f32_host,
+                    void* workspace, int64_t workspace_bytes, void* stream);
+
+/* ---- Roofline denominator: measures this GPU's 32-bit population-count issue rate with a
+ * register-only loop (no memory traffic) and the SM clock it ran at.  Synchronous.
+ * popc_per_s: lane-level POPC results per second over the whole chip; sm_mhz: SM clock
+ * observed inside the kernel; sms: multiprocessor count.  Any pointer may be NULL. */
+int mpq_measure_popc_peak(double* popc_per_s, double* sm_mhz, int* sms, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MPQ_H_ */

@@ -1,0 +1,208 @@
+"""Thin Python binding of libmpq.so: argument marshalling only.
+
+Every function has the name and the argument order of its C entry point in
+``include/mpq.h`` (minus the ``mpq_`` prefix) and takes torch CUDA tensors where
+the C side takes device pointers.  torch is used for device memory and streams
+only; every step of the path runs in the library's own kernels.  There is no CPU
+fallback: if the library is missing or a call fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libmpq.so")
+
+OK = 0
+SCALE_PER_TENSOR, SCALE_PER_ROW = 0, 1
+ACT_HTANH, ACT_HRELU = 0, 1
+
+_lib = None
+
+
+class MpqError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__("%s failed: %s (status %d)" % (where, status_string(status), status))
+
+
+def lib() -> ctypes.CDLL:
+    """Loads libmpq.so (must have been built in-tree, see ``build.py``)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError("libmpq.so is not built: run `python -m paper_1905_13389_b200.build` "
+                              "(there is no CPU fallback)")
+        L = ctypes.CDLL(LIB_PATH)
+        i64, i32, P = ctypes.c_int64, ctypes.c_int, ctypes.c_void_p
+        L.mpq_status_string.argtypes = [i32]
+        L.mpq_status_string.restype = ctypes.c_char_p
+        L.mpq_row_words.argtypes = [i64]
+        L.mpq_row_words.restype = i64
+        L.mpq_packed_words.argtypes = [i64, i64, i32]
+        L.mpq_packed_words.restype = i64
+        L.mpq_absmax.argtypes = [P, i64, i64, i64, i32, i32, P, P]
+        L.mpq_encode.argtypes = [P, i64, i64, i64, P, i32, i32, i32, P, P]
+        L.mpq_encode_nchw.argtypes = [P, i32, i32, i32, i32, P, i32, i32, P, P]
+        L.mpq_encode_oihw.argtypes = [P, i32, i32, i32, i32, P, i32, i32, P, P, P]
+        L.mpq_gemm.argtypes = [P, i32, P, i32, i64, i64, i64, P, P, i64, P, P, i32, P]
+        L.mpq_conv.argtypes = [P, i32, i32, i32, i32, i32, P, i32, P, i32, i32, i32, i32, i32, P, P, P, P, i32, P]
+        L.mpq_add_relu.argtypes = [P, P, P, i64, P]
+        L.mpq_linear_host_workspace.argtypes = [i64, i64, i64, i32, i32]
+        L.mpq_linear_host_workspace.restype = i64
+        L.mpq_linear_host.argtypes = [P, P, i64, i64, i64, i32, i32, i32, i32, P, P, P, i64, P]
+        L.mpq_measure_popc_peak.argtypes = [ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double),
+                                            ctypes.POINTER(ctypes.c_int), P]
+        for name in ("mpq_absmax", "mpq_encode", "mpq_encode_nchw", "mpq_encode_oihw", "mpq_gemm", "mpq_conv",
+                     "mpq_add_relu", "mpq_linear_host", "mpq_measure_popc_peak"):
+            getattr(L, name).restype = i32
+        _lib = L
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return lib().mpq_status_string(int(status)).decode()
+
+
+def row_words(k: int) -> int:
+    return int(lib().mpq_row_words(k))
+
+
+def packed_words(rows: int, k: int, bits: int) -> int:
+    return int(lib().mpq_packed_words(rows, k, bits))
+
+
+def _check(status: int, where: str):
+    if status != OK:
+        raise MpqError(status, where)
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _ptr(t: Optional[torch.Tensor], dtype=None) -> Optional[int]:
+    if t is None:
+        return None
+    if not t.is_cuda:
+        raise ValueError("expected a CUDA tensor")
+    if dtype is not None and t.dtype != dtype:
+        raise ValueError("expected dtype %s, got %s" % (dtype, t.dtype))
+    if not t.is_contiguous():
+        raise ValueError("expected a contiguous tensor")
+    return t.data_ptr()
+
+
+def absmax(x: torch.Tensor, mode: int = SCALE_PER_TENSOR, act: int = ACT_HTANH,
+           out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """Range of a float tensor viewed as [rows x k] (rows = leading axis): 1 or rows values."""
+    rows = x.shape[0]
+    k = x.numel() // rows
+    if out is None:
+        out = torch.empty(rows if mode == SCALE_PER_ROW else 1, dtype=torch.float32, device=x.device)
+    _check(lib().mpq_absmax(_ptr(x, torch.float32), rows, k, k, mode, act, _ptr(out, torch.float32), _stream()),
+           "mpq_absmax")
+    return out
+
+
+def encode(x: torch.Tensor, scale: torch.Tensor, bits: int, mode: int = SCALE_PER_TENSOR,
+           act: int = ACT_HTANH, out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """[rows x k] fp32 -> planes [bits][rows][row_words(k)] (int32 storage of the uint32 words)."""
+    rows, k = x.shape
+    if out is None:
+        out = torch.empty((bits, rows, row_words(k)), dtype=torch.int32, device=x.device)
+    _check(lib().mpq_encode(_ptr(x, torch.float32), rows, k, k, _ptr(scale, torch.float32), mode, act, bits,
+                            _ptr(out, torch.int32), _stream()), "mpq_encode")
+    return out
+
+
+def encode_nchw(x: torch.Tensor, scale: torch.Tensor, bits: int, act: int = ACT_HTANH,
+                out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """[N][C][H][W] fp32 -> planes [bits][N][H][W][C/32]."""
+    N, C, H, W = x.shape
+    if out is None:
+        out = torch.empty((bits, N, H, W, max(C // 32, 1)), dtype=torch.int32, device=x.device)
+    _check(lib().mpq_encode_nchw(_ptr(x, torch.float32), N, C, H, W, _ptr(scale, torch.float32), act, bits,
+                                 _ptr(out, torch.int32), _stream()), "mpq_encode_nchw")
+    return out
+
+
+def encode_oihw(w: torch.Tensor, scale: torch.Tensor, bits: int, mode: int = SCALE_PER_ROW):
+    """[O][C][KH][KW] fp32 -> (planes [bits][O][row_words(KH*KW*C)], tap_sums [KH*KW][O])."""
+    O, C, KH, KW = w.shape
+    planes = torch.empty((bits, O, row_words(KH * KW * C)), dtype=torch.int32, device=w.device)
+    tap_sums = torch.empty((KH * KW, O), dtype=torch.int32, device=w.device)
+    _check(lib().mpq_encode_oihw(_ptr(w, torch.float32), O, C, KH, KW, _ptr(scale, torch.float32), mode, bits,
+                                 _ptr(planes, torch.int32), _ptr(tap_sums, torch.int32), _stream()),
+           "mpq_encode_oihw")
+    return planes, tap_sums
+
+
+def gemm(a_planes: torch.Tensor, a_bits: int, b_planes: torch.Tensor, b_bits: int, m: int, n: int, k: int,
+         c_i32: Optional[torch.Tensor] = None, c_f32: Optional[torch.Tensor] = None,
+         a_scale: Optional[torch.Tensor] = None, b_scale: Optional[torch.Tensor] = None,
+         b_mode: int = SCALE_PER_TENSOR):
+    """C = A B^T on packed planes; writes the int32 accumulators and/or the scaled fp32 output."""
+    ldc = n
+    _check(lib().mpq_gemm(_ptr(a_planes, torch.int32), a_bits, _ptr(b_planes, torch.int32), b_bits, m, n, k,
+                          _ptr(c_i32, torch.int32), _ptr(c_f32, torch.float32), ldc,
+                          _ptr(a_scale, torch.float32), _ptr(b_scale, torch.float32), b_mode, _stream()),
+           "mpq_gemm")
+    return c_i32, c_f32
+
+
+def conv(x_planes: torch.Tensor, a_bits: int, N: int, C: int, H: int, W: int,
+         w_planes: torch.Tensor, w_bits: int, tap_sums: Optional[torch.Tensor],
+         O: int, KH: int, KW: int, stride: int, pad: int,
+         y_i32: Optional[torch.Tensor] = None, y_f32: Optional[torch.Tensor] = None,
+         x_scale: Optional[torch.Tensor] = None, w_scale: Optional[torch.Tensor] = None,
+         w_mode: int = SCALE_PER_ROW):
+    """Implicit-im2col convolution on packed planes; y is [N][O][Ho][Wo]."""
+    _check(lib().mpq_conv(_ptr(x_planes, torch.int32), a_bits, N, C, H, W, _ptr(w_planes, torch.int32), w_bits,
+                          _ptr(tap_sums, torch.int32), O, KH, KW, stride, pad,
+                          _ptr(y_i32, torch.int32), _ptr(y_f32, torch.float32),
+                          _ptr(x_scale, torch.float32), _ptr(w_scale, torch.float32), w_mode, _stream()),
+           "mpq_conv")
+    return y_i32, y_f32
+
+
+def add_relu(a: torch.Tensor, b: Optional[torch.Tensor], y: torch.Tensor) -> torch.Tensor:
+    _check(lib().mpq_add_relu(_ptr(a, torch.float32), _ptr(b, torch.float32), _ptr(y, torch.float32),
+                              a.numel(), _stream()), "mpq_add_relu")
+    return y
+
+
+def linear_host_workspace(m: int, n: int, k: int, a_bits: int, w_bits: int) -> int:
+    return int(lib().mpq_linear_host_workspace(m, n, k, a_bits, w_bits))
+
+
+def linear_host(x_host: torch.Tensor, w_host: torch.Tensor, a_bits: int, w_bits: int,
+                a_act: int = ACT_HTANH, w_mode: int = SCALE_PER_TENSOR,
+                out_i32_host: Optional[torch.Tensor] = None, out_f32_host: Optional[torch.Tensor] = None,
+                workspace: Optional[torch.Tensor] = None):
+    """Whole encoded fully-connected layer from (pinned) host tensors; synchronizes the stream."""
+    m, k = x_host.shape
+    n, _ = w_host.shape
+    need = linear_host_workspace(m, n, k, a_bits, w_bits)
+    if workspace is None:
+        workspace = torch.empty(need, dtype=torch.uint8, device="cuda")
+    for t in (x_host, w_host, out_i32_host, out_f32_host):
+        if t is not None and (t.is_cuda or not t.is_contiguous()):
+            raise ValueError("host tensors must be contiguous CPU tensors")
+    hp = lambda t: None if t is None else t.data_ptr()
+    _check(lib().mpq_linear_host(hp(x_host), hp(w_host), m, n, k, a_bits, w_bits, a_act, w_mode,
+                                 hp(out_i32_host), hp(out_f32_host), workspace.data_ptr(), workspace.numel(),
+                                 _stream()), "mpq_linear_host")
+    return out_i32_host, out_f32_host
+
+
+def measure_popc_peak():
+    """(lane-level POPC results per second over the chip, SM MHz seen by the probe, SM count)."""
+    rate, mhz, sms = ctypes.c_double(), ctypes.c_double(), ctypes.c_int()
+    _check(lib().mpq_measure_popc_peak(ctypes.byref(rate), ctypes.byref(mhz), ctypes.byref(sms), _stream()),
+           "mpq_measure_popc_peak")
+    return rate.value, mhz.value, sms.value

@@ -1,0 +1,146 @@
+// Status strings, size queries, the host-buffer fully-connected layer and the POPC-rate probe.
+#include "mpq_common.cuh"
+
+using namespace mpq;
+
+extern "C" const char* mpq_status_string(int status) {
+    switch (status) {
+        case MPQ_OK: return "ok";
+        case MPQ_ERR_NULL: return "null pointer";
+        case MPQ_ERR_BAD_SHAPE: return "bad shape";
+        case MPQ_ERR_UNSUPPORTED: return "unsupported configuration";
+        case MPQ_ERR_OVERFLOW: return "int32 accumulator would overflow";
+        case MPQ_ERR_ALIGN: return "pointer not 16-byte aligned";
+        case MPQ_ERR_CUDA: return "CUDA runtime error";
+        case MPQ_ERR_WORKSPACE: return "workspace too small";
+    }
+    return "unknown status";
+}
+
+extern "C" int64_t mpq_row_words(int64_t k) { return k > 0 ? row_words(k) : 0; }
+
+extern "C" int64_t mpq_packed_words(int64_t rows, int64_t k, int bits) {
+    if (rows <= 0 || k <= 0 || !bits_ok(bits)) return 0;
+    return (int64_t)bits * rows * row_words(k);
+}
+
+// ---- host-buffer fully-connected layer -----------------------------------------------------
+namespace {
+struct LinearLayout {
+    int64_t x, w, s_a, s_w, a_planes, w_planes, out_i32, out_f32, total;
+};
+inline int64_t up256(int64_t v) { return (v + 255) / 256 * 256; }
+LinearLayout linear_layout(int64_t m, int64_t n, int64_t k, int a_bits, int w_bits) {
+    LinearLayout L;
+    int64_t off = 0;
+    L.x = off; off += up256(m * k * 4);
+    L.w = off; off += up256(n * k * 4);
+    L.s_a = off; off += 256;
+    L.s_w = off; off += up256(n * 4);
+    L.a_planes = off; off += up256(mpq_packed_words(m, k, a_bits) * 4);
+    L.w_planes = off; off += up256(mpq_packed_words(n, k, w_bits) * 4);
+    L.out_i32 = off; off += up256(m * n * 4);
+    L.out_f32 = off; off += up256(m * n * 4);
+    L.total = off;
+    return L;
+}
+}  // namespace
+
+extern "C" int64_t mpq_linear_host_workspace(int64_t m, int64_t n, int64_t k, int a_bits, int w_bits) {
+    if (m <= 0 || n <= 0 || k <= 0 || !bits_ok(a_bits) || !bits_ok(w_bits)) return 0;
+    return linear_layout(m, n, k, a_bits, w_bits).total;
+}
+
+extern "C" int mpq_linear_host(const float* x_host, const float* w_host, int64_t m, int64_t n, int64_t k,
+                               int a_bits, int w_bits, int a_act, int w_mode,
+                               int32_t* out_i32_host, float* out_f32_host,
+                               void* workspace, int64_t workspace_bytes, void* stream) {
+    if (!x_host || !w_host || !workspace || (!out_i32_host && !out_f32_host)) return MPQ_ERR_NULL;
+    if (m <= 0 || n <= 0 || k <= 0) return MPQ_ERR_BAD_SHAPE;
+    if (!bits_ok(a_bits) || !bits_ok(w_bits)) return MPQ_ERR_UNSUPPORTED;
+    if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return MPQ_ERR_ALIGN;
+    const LinearLayout L = linear_layout(m, n, k, a_bits, w_bits);
+    if (workspace_bytes < L.total) return MPQ_ERR_WORKSPACE;
+    cudaStream_t st = (cudaStream_t)stream;
+    char* ws = static_cast<char*>(workspace);
+    float* x = reinterpret_cast<float*>(ws + L.x);
+    float* w = reinterpret_cast<float*>(ws + L.w);
+    float* s_a = reinterpret_cast<float*>(ws + L.s_a);
+    float* s_w = reinterpret_cast<float*>(ws + L.s_w);
+    uint32_t* ap = reinterpret_cast<uint32_t*>(ws + L.a_planes);
+    uint32_t* wp = reinterpret_cast<uint32_t*>(ws + L.w_planes);
+    int32_t* oi = reinterpret_cast<int32_t*>(ws + L.out_i32);
+    float* of = reinterpret_cast<float*>(ws + L.out_f32);
+
+    if (cudaMemcpyAsync(x, x_host, (size_t)m * k * 4, cudaMemcpyHostToDevice, st) != cudaSuccess) return MPQ_ERR_CUDA;
+    if (cudaMemcpyAsync(w, w_host, (size_t)n * k * 4, cudaMemcpyHostToDevice, st) != cudaSuccess) return MPQ_ERR_CUDA;
+    int rc;
+    if ((rc = mpq_absmax(x, m, k, k, MPQ_SCALE_PER_TENSOR, a_act, s_a, st)) != MPQ_OK) return rc;
+    if ((rc = mpq_absmax(w, n, k, k, w_mode, MPQ_ACT_HTANH, s_w, st)) != MPQ_OK) return rc;
+    if ((rc = mpq_encode(x, m, k, k, s_a, MPQ_SCALE_PER_TENSOR, a_act, a_bits, ap, st)) != MPQ_OK) return rc;
+    if ((rc = mpq_encode(w, n, k, k, s_w, w_mode, MPQ_ACT_HTANH, w_bits, wp, st)) != MPQ_OK) return rc;
+    if ((rc = mpq_gemm(ap, a_bits, wp, w_bits, m, n, k, out_i32_host ? oi : nullptr, out_f32_host ? of : nullptr, n,
+                       s_a, s_w, w_mode, st)) != MPQ_OK) return rc;
+    if (out_i32_host && cudaMemcpyAsync(out_i32_host, oi, (size_t)m * n * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess) return MPQ_ERR_CUDA;
+    if (out_f32_host && cudaMemcpyAsync(out_f32_host, of, (size_t)m * n * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess) return MPQ_ERR_CUDA;
+    return cudaStreamSynchronize(st) == cudaSuccess ? MPQ_OK : MPQ_ERR_CUDA;
+}
+
+// ---- POPC issue-rate probe ----------------------------------------------------------------
+namespace {
+constexpr int kProbeChains = 8;
+// The probe's few result words live in the module so that the call needs no buffer from the caller.
+__device__ unsigned long long probe_clk[2];
+__device__ uint32_t probe_sink[1];
+__global__ void popc_rate_kernel(uint32_t seed, int iters, uint32_t* sink, unsigned long long* clk) {
+    uint32_t x[kProbeChains];
+    const uint32_t s = seed ^ (threadIdx.x * 0x9E3779B9u);
+#pragma unroll
+    for (int i = 0; i < kProbeChains; ++i) x[i] = s * (uint32_t)(i + 3);
+    unsigned long long g0, g1;
+    const long long c0 = clock64();
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(g0));
+    for (int it = 0; it < iters; ++it) {
+#pragma unroll
+        for (int i = 0; i < kProbeChains; ++i) x[i] = __popc(x[i]) + s;   // independent chains
+    }
+    const long long c1 = clock64();
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(g1));
+    uint32_t r = 0;
+#pragma unroll
+    for (int i = 0; i < kProbeChains; ++i) r += x[i];
+    if (r == 0xFFFFFFFFu) sink[0] = r;          // never true: keeps the loop alive
+    if (threadIdx.x == 0 && blockIdx.x == 0) { clk[0] = (unsigned long long)(c1 - c0); clk[1] = g1 - g0; }
+}
+}  // namespace
+
+extern "C" int mpq_measure_popc_peak(double* popc_per_s, double* sm_mhz, int* sms, void* stream) {
+    cudaStream_t st = (cudaStream_t)stream;
+    int dev = 0, n_sm = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return MPQ_ERR_CUDA;
+    if (cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return MPQ_ERR_CUDA;
+    unsigned long long* d_clk = nullptr; uint32_t* d_sink = nullptr;
+    if (cudaGetSymbolAddress((void**)&d_clk, probe_clk) != cudaSuccess) return MPQ_ERR_CUDA;
+    if (cudaGetSymbolAddress((void**)&d_sink, probe_sink) != cudaSuccess) return MPQ_ERR_CUDA;
+    const int threads = 512, blocks_per_sm = 2, iters = 20000;
+    cudaEvent_t e0, e1;
+    if (cudaEventCreate(&e0) != cudaSuccess || cudaEventCreate(&e1) != cudaSuccess) return MPQ_ERR_CUDA;
+    float best_ms = 1e30f; unsigned long long h_clk[2] = {0, 0}, best_clk[2] = {1, 1};
+    int rc = MPQ_OK;
+    for (int rep = 0; rep < 4 && rc == MPQ_OK; ++rep) {
+        cudaEventRecord(e0, st);
+        popc_rate_kernel<<<n_sm * blocks_per_sm, threads, 0, st>>>(12345u + rep, iters, d_sink, d_clk);
+        cudaEventRecord(e1, st);
+        if (cudaEventSynchronize(e1) != cudaSuccess || cudaGetLastError() != cudaSuccess) { rc = MPQ_ERR_CUDA; break; }
+        float ms = 0; cudaEventElapsedTime(&ms, e0, e1);
+        if (cudaMemcpy(h_clk, d_clk, sizeof(h_clk), cudaMemcpyDeviceToHost) != cudaSuccess) { rc = MPQ_ERR_CUDA; break; }
+        if (rep > 0 && ms < best_ms) { best_ms = ms; best_clk[0] = h_clk[0]; best_clk[1] = h_clk[1]; }
+    }
+    cudaEventDestroy(e0); cudaEventDestroy(e1);
+    if (rc != MPQ_OK) return rc;
+    const double popcs = (double)n_sm * blocks_per_sm * threads * (double)iters * kProbeChains;
+    if (popc_per_s) *popc_per_s = popcs / (best_ms * 1e-3);
+    if (sm_mhz) *sm_mhz = (double)best_clk[0] / (double)best_clk[1] * 1e3;
+    if (sms) *sms = n_sm;
+    return MPQ_OK;
+}

@@ -1,0 +1,320 @@
+// Branch-fused binary GEMM / implicit-im2col convolution on packed {-1,+1} bit-planes.
+//
+// One kernel computes, for a tile of outputs, ALL a_bits x w_bits binary-branch products of
+// Eq. 7-10 at once: every bit-plane of the two operand tiles is staged once in shared memory
+// (cp.async, multi-stage ring) and each thread accumulates
+//     S[r][c] = sum_{i,j} 2^(i+j) * popcount(A_i[r] xor B_j[c])
+// for a small register tile of outputs, then applies the decoder
+//     acc = L_a L_w k - 2 S,   out = float(acc) * alpha[c]           (Eq. 18)
+// in the store.  The arithmetic is XOR + POPC + shift-add on the integer pipes: the B200's
+// 5th-generation tensor cores have no 1-bit kind, and the legacy 1-bit mma.sync form measured
+// slower than the POPC pipe on this chip.
+//
+// Roles.  The "held" operand (HB planes, TH items per thread) lives in registers as 128-bit
+// k-quads; the "streamed" operand (SB planes, TS items per thread) is read quad by quad from
+// shared memory.  Threads form a 16 x 16 grid: ty indexes held items, tx streamed items, so
+// streamed reads are conflict-free 16-byte accesses and held reads are broadcasts.
+//   GEMM mode: held = A rows (activations), streamed = B rows (weights / output columns).
+//   CONV mode: held = weight rows (output channels), streamed = output pixels, gathered on the
+//              fly from planes[bits][N][H][W][C/32]; consecutive tx = consecutive pixels, which
+//              is the contiguous direction of the NCHW output.
+#pragma once
+#include "mpq_common.cuh"
+
+namespace mpq {
+
+enum { kModeGemm = 0, kModeConv = 1 };
+
+struct BranchParams {
+    const uint32_t* held;      // GEMM: A planes [HB][m][rw];      CONV: weight planes [HB][O][rw]
+    const uint32_t* streamed;  // GEMM: B planes [SB][n][rw];      CONV: x planes [SB][N][H][W][Cw]
+    int64_t held_rows;         // GEMM: m;  CONV: O
+    int64_t streamed_rows;     // GEMM: n;  CONV: N*Ho*Wo
+    int64_t rw;                // words per packed row (GEMM: both operands; CONV: weight rows)
+    int64_t k;                 // elements per dot product (CONV: KH*KW*C)
+    int32_t* out_i32;
+    float* out_f32;
+    int64_t ldc;               // GEMM only
+    const float* a_scale;      // activation range, 1 value (may be null when out_f32 is null)
+    const float* w_scale;      // weight range, 1 or per-output-channel values
+    int w_per_row;
+    // CONV only
+    int N, C, H, W, O, KH, KW, stride, pad, Ho, Wo, Cw;
+    int granule;               // words gathered per copy: 1 (C=32), 2 (C=64) or 4 (C % 128 == 0)
+    const int32_t* tap_sums;   // [KH*KW][O]
+};
+
+__device__ __forceinline__ void cp_async_16(void* smem_dst, const void* gsrc, bool valid) {
+    const unsigned dst = (unsigned)__cvta_generic_to_shared(smem_dst);
+    const int src_bytes = valid ? 16 : 0;   // 0 => the 16 bytes are zero-filled
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(dst), "l"(gsrc), "r"(src_bytes) : "memory");
+}
+template <int BYTES>
+__device__ __forceinline__ void cp_async_small(void* smem_dst, const void* gsrc, bool valid) {
+    const unsigned dst = (unsigned)__cvta_generic_to_shared(smem_dst);
+    const int src_bytes = valid ? BYTES : 0;
+    asm volatile("cp.async.ca.shared.global [%0], [%1], %2, %3;\n" ::"r"(dst), "l"(gsrc), "n"(BYTES), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory"); }
+
+__device__ __forceinline__ int popc_xor4(const uint4& a, const uint4& b) {
+    return __popc(a.x ^ b.x) + __popc(a.y ^ b.y) + __popc(a.z ^ b.z) + __popc(a.w ^ b.w);
+}
+
+template <int HB, int SB>
+struct BranchTile {
+    static constexpr int TH = (HB == 1) ? 8 : (HB == 2) ? 4 : (HB <= 4) ? 2 : 1;   // TH*HB <= 8 quads held
+    static constexpr int KQ = (SB == 1) ? 8 : (SB == 2) ? 4 : (SB <= 4) ? 2 : 1;   // k-quads per stage
+    static constexpr int STAGES = 3;
+    static constexpr int THREADS = 256;
+};
+
+template <int HB, int SB, int TS, int MODE>
+__global__ void __launch_bounds__(256, 2)
+branch_kernel(const BranchParams p) {
+    using T = BranchTile<HB, SB>;
+    constexpr int TH = T::TH, KQ = T::KQ, STAGES = T::STAGES;
+    constexpr int BH = 16 * TH, BS = 16 * TS;
+    constexpr int H_QUADS = HB * KQ * BH;          // 16-byte chunks per stage, held operand
+    constexpr int S_QUADS = SB * KQ * BS;          // ... streamed operand
+    constexpr int STAGE_QUADS = H_QUADS + S_QUADS;
+
+    extern __shared__ uint4 smem[];
+    __shared__ int row_n[MODE == kModeConv ? BS : 1];      // image index, or -1 for rows past the end
+    __shared__ int row_ih0[MODE == kModeConv ? BS : 1];    // top-left input coordinate of the window
+    __shared__ int row_iw0[MODE == kModeConv ? BS : 1];
+
+    const int tid = threadIdx.x;
+    const int tx = tid & 15, ty = tid >> 4;
+    const int64_t s_tiles = ceil_div(p.streamed_rows, BS);
+    const int64_t s0 = (int64_t)(blockIdx.x % s_tiles) * BS;
+    const int64_t h0 = (int64_t)(blockIdx.x / s_tiles) * BH;
+    const int64_t kq_total = p.rw / 4;
+    const int n_iters = (int)ceil_div(kq_total, KQ);
+
+    if (MODE == kModeConv) {
+        for (int r = tid; r < BS; r += 256) {
+            const int64_t g = s0 + r;
+            if (g < p.streamed_rows) {
+                const int64_t hw = (int64_t)p.Ho * p.Wo;
+                const int n = (int)(g / hw);
+                const int rem = (int)(g % hw);
+                row_n[r] = n;
+                row_ih0[r] = (rem / p.Wo) * p.stride - p.pad;
+                row_iw0[r] = (rem % p.Wo) * p.stride - p.pad;
+            } else {
+                row_n[r] = -1; row_ih0[r] = 0; row_iw0[r] = 0;
+            }
+        }
+        __syncthreads();
+    }
+
+    auto load_stage = [&](int stage, int64_t kq0) {
+        uint4* hs = smem + (size_t)stage * STAGE_QUADS;
+        uint4* ss = hs + H_QUADS;
+        // held operand: [plane][kq][row], consecutive threads -> consecutive kq of one row
+#pragma unroll
+        for (int base = 0; base < H_QUADS; base += 256) {
+            const int id = base + tid;
+            if (H_QUADS % 256 == 0 || id < H_QUADS) {
+                const int kq = id % KQ, row = (id / KQ) % BH, plane = id / (KQ * BH);
+                const int64_t grow = h0 + row, gkq = kq0 + kq;
+                const bool ok = grow < p.held_rows && gkq < kq_total;
+                const uint32_t* src = ok ? p.held + ((int64_t)plane * p.held_rows + grow) * p.rw + gkq * 4 : p.held;
+                cp_async_16(hs + (plane * KQ + kq) * BH + row, src, ok);
+            }
+        }
+        if (MODE == kModeGemm) {
+#pragma unroll
+            for (int base = 0; base < S_QUADS; base += 256) {
+                const int id = base + tid;
+                if (S_QUADS % 256 == 0 || id < S_QUADS) {
+                    const int kq = id % KQ, row = (id / KQ) % BS, plane = id / (KQ * BS);
+                    const int64_t grow = s0 + row, gkq = kq0 + kq;
+                    const bool ok = grow < p.streamed_rows && gkq < kq_total;
+                    const uint32_t* src = ok ? p.streamed + ((int64_t)plane * p.streamed_rows + grow) * p.rw + gkq * 4 : p.streamed;
+                    cp_async_16(ss + (plane * KQ + kq) * BS + row, src, ok);
+                }
+            }
+        } else {
+            // implicit im2col: one copy = `granule` words of one tap of one pixel (never crosses a tap)
+            const int G = p.granule;
+            const int parts = 4 / G;
+            const int granules = S_QUADS * parts;
+            const int taps = p.KH * p.KW;
+            for (int id = tid; id < granules; id += 256) {
+                const int part = id % parts, kq = (id / parts) % KQ;
+                const int row = (id / (parts * KQ)) % BS, plane = id / (parts * KQ * BS);
+                const int64_t kword = (kq0 + kq) * 4 + part * G;
+                const int tap = (int)(kword / p.Cw), cw = (int)(kword % p.Cw);
+                const int n = row_n[row];
+                const int ih = row_ih0[row] + tap / p.KW, iw = row_iw0[row] + tap % p.KW;
+                const bool ok = n >= 0 && tap < taps && ih >= 0 && ih < p.H && iw >= 0 && iw < p.W;
+                const uint32_t* src = ok ? p.streamed + ((((int64_t)plane * p.N + n) * p.H + ih) * p.W + iw) * p.Cw + cw
+                                         : p.streamed;
+                uint32_t* dst = reinterpret_cast<uint32_t*>(ss + (plane * KQ + kq) * BS + row) + part * G;
+                if (G == 4) cp_async_16(dst, src, ok);
+                else if (G == 2) cp_async_small<8>(dst, src, ok);
+                else cp_async_small<4>(dst, src, ok);
+            }
+        }
+    };
+
+    uint32_t acc[TH][TS];
+#pragma unroll
+    for (int a = 0; a < TH; ++a)
+#pragma unroll
+        for (int b = 0; b < TS; ++b) acc[a][b] = 0u;
+
+#pragma unroll
+    for (int s = 0; s < STAGES - 1; ++s) {
+        if (s < n_iters) load_stage(s, (int64_t)s * KQ);
+        cp_async_commit();
+    }
+
+    for (int it = 0; it < n_iters; ++it) {
+        cp_async_wait<STAGES - 2>();
+        __syncthreads();
+        {
+            const int nxt = it + STAGES - 1;
+            if (nxt < n_iters) load_stage(nxt % STAGES, (int64_t)nxt * KQ);
+            cp_async_commit();
+        }
+        const uint4* hs = smem + (size_t)(it % STAGES) * STAGE_QUADS;
+        const uint4* ss = hs + H_QUADS;
+#pragma unroll
+        for (int kq = 0; kq < KQ; ++kq) {
+            uint4 h[TH][HB];
+#pragma unroll
+            for (int a = 0; a < TH; ++a)
+#pragma unroll
+                for (int i = 0; i < HB; ++i) h[a][i] = hs[(i * KQ + kq) * BH + ty + 16 * a];
+#pragma unroll
+            for (int b = 0; b < TS; ++b) {
+#pragma unroll
+                for (int j = 0; j < SB; ++j) {
+                    const uint4 s = ss[(j * KQ + kq) * BS + tx + 16 * b];
+#pragma unroll
+                    for (int a = 0; a < TH; ++a)
+#pragma unroll
+                        for (int i = 0; i < HB; ++i)
+                            acc[a][b] += (uint32_t)popc_xor4(h[a][i], s) << (i + j);
+                }
+            }
+        }
+    }
+    cp_async_wait<0>();
+
+    // ---- decoder: acc = L_a L_w k - 2 S, then the fused scale of Eq. 18 -------------------
+    constexpr uint32_t LL = (uint32_t)(((1 << HB) - 1) * ((1 << SB) - 1));
+    const uint32_t full = LL * (uint32_t)p.k;
+    const bool want_f32 = p.out_f32 != nullptr;
+    // activation bits: GEMM held = A; CONV streamed = x
+    constexpr int A_BITS = (MODE == kModeGemm) ? HB : SB;
+    constexpr int W_BITS = (MODE == kModeGemm) ? SB : HB;
+    float fa = 0.0f;
+    if (want_f32) fa = __fdiv_rn(__ldg(p.a_scale), (float)((1 << A_BITS) - 1));
+    const float Lw = (float)((1 << W_BITS) - 1);
+
+    if (MODE == kModeGemm) {
+#pragma unroll
+        for (int b = 0; b < TS; ++b) {
+            const int64_t col = s0 + tx + 16 * b;
+            if (col >= p.streamed_rows) continue;
+            float alpha = 0.0f;
+            if (want_f32) alpha = __fmul_rn(fa, __fdiv_rn(__ldg(p.w_scale + (p.w_per_row ? col : 0)), Lw));
+#pragma unroll
+            for (int a = 0; a < TH; ++a) {
+                const int64_t row = h0 + ty + 16 * a;
+                if (row >= p.held_rows) continue;
+                const int32_t v = (int32_t)(full - 2u * acc[a][b]);
+                if (p.out_i32) p.out_i32[row * p.ldc + col] = v;
+                if (want_f32) p.out_f32[row * p.ldc + col] = __fmul_rn((float)v, alpha);
+            }
+        }
+    } else {
+        const int taps = p.KH * p.KW;
+        const int64_t hw = (int64_t)p.Ho * p.Wo;
+        float alpha[TH];
+#pragma unroll
+        for (int a = 0; a < TH; ++a) {
+            const int64_t o = h0 + ty + 16 * a;
+            alpha[a] = 0.0f;
+            if (want_f32 && o < p.held_rows)
+                alpha[a] = __fmul_rn(fa, __fdiv_rn(__ldg(p.w_scale + (p.w_per_row ? o : 0)), Lw));
+        }
+#pragma unroll
+        for (int b = 0; b < TS; ++b) {
+            const int r = tx + 16 * b;
+            const int n = row_n[r];
+            if (n < 0) continue;
+            const int ih0 = row_ih0[r], iw0 = row_iw0[r];
+            // taps of this pixel that fall outside the image were staged as all-zero bits, i.e. as the
+            // code -L_a; what they added, -L_a * tap_sum[tap][o], is taken out again so they count as 0
+            unsigned outside = 0;
+            if (p.pad > 0) {
+                for (int t = 0; t < taps; ++t) {
+                    const int ih = ih0 + t / p.KW, iw = iw0 + t % p.KW;
+                    if (ih < 0 || ih >= p.H || iw < 0 || iw >= p.W) outside |= 1u << t;
+                }
+            }
+            const int64_t rem = (s0 + r) % hw;
+#pragma unroll
+            for (int a = 0; a < TH; ++a) {
+                const int64_t o = h0 + ty + 16 * a;
+                if (o >= p.held_rows) continue;
+                int32_t v = (int32_t)(full - 2u * acc[a][b]);
+                if (outside) {
+                    int32_t fix = 0;
+                    for (int t = 0; t < taps; ++t)
+                        if (outside & (1u << t)) fix += __ldg(p.tap_sums + (int64_t)t * p.O + o);
+                    v += ((1 << A_BITS) - 1) * fix;
+                }
+                const int64_t idx = ((int64_t)n * p.O + o) * hw + rem;
+                if (p.out_i32) p.out_i32[idx] = v;
+                if (want_f32) p.out_f32[idx] = __fmul_rn((float)v, alpha[a]);
+            }
+        }
+    }
+}
+
+template <int HB, int SB, int TS, int MODE>
+static int launch_branch(const BranchParams& p, cudaStream_t st) {
+    using T = BranchTile<HB, SB>;
+    constexpr int BH = 16 * T::TH, BS = 16 * TS;
+    constexpr size_t smem_bytes = (size_t)T::STAGES * (HB * T::KQ * BH + SB * T::KQ * BS) * sizeof(uint4);
+    auto kern = branch_kernel<HB, SB, TS, MODE>;
+    static bool configured = false;   // per instantiation; attribute is per function, set once per process+device
+    static int configured_dev = -1;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return MPQ_ERR_CUDA;
+    if (!configured || configured_dev != dev) {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes) != cudaSuccess)
+            return MPQ_ERR_CUDA;
+        configured = true; configured_dev = dev;
+    }
+    const int64_t blocks = ceil_div(p.streamed_rows, BS) * ceil_div(p.held_rows, BH);
+    if (blocks <= 0 || blocks > 0x7fffffffLL) return MPQ_ERR_BAD_SHAPE;
+    kern<<<(unsigned)blocks, 256, smem_bytes, st>>>(p);
+    return launch_status();
+}
+
+// Streamed-side tile width: 128 columns normally, 32 when the wide tile would leave most of the
+// 148 SMs idle (skinny problems such as a batch-64 fully-connected layer).
+template <int HB, int SB>
+static int launch_gemm_auto(const BranchParams& p, cudaStream_t st) {
+    using T = BranchTile<HB, SB>;
+    const int64_t wide = ceil_div(p.streamed_rows, 128) * ceil_div(p.held_rows, 16 * T::TH);
+    if (wide >= 148) return launch_branch<HB, SB, 8, kModeGemm>(p, st);
+    return launch_branch<HB, SB, 2, kModeGemm>(p, st);
+}
+
+// One translation unit per held-operand width instantiates all eight streamed widths.
+template <int HB>
+int launch_gemm_hb(int sb, const BranchParams& p, cudaStream_t st);
+template <int HB>
+int launch_conv_hb(int sb, const BranchParams& p, cudaStream_t st);
+
+}  // namespace mpq

@@ -1,0 +1,333 @@
+// Range (max-abs) and Encoder kernels: fp32 -> packed {-1,+1} bit-planes.
+//
+// Encoder = quantizer of Eq. 15 (round half up) + the code of Table 2 / Eq. 10, stored one bit
+// per element.  All three layouts are HBM-bound: 4 bytes read and bits/8 bytes written per
+// element, so the kernels are organised around coalesced reads with many loads in flight.
+#include "mpq_common.cuh"
+
+namespace mpq {
+
+// ------------------------------------------------------------------------------------------
+// Range: max |x| (HTanh) or max of the positive side (HReLU); NaNs are ignored by fmaxf.
+// Non-negative floats order like their bit patterns, so the cross-CTA step is an integer atomicMax.
+// ------------------------------------------------------------------------------------------
+constexpr int kAbsmaxThreads = 256;
+constexpr int kAbsmaxChunk = 8192;  // elements per CTA
+
+template <int ACT, bool VEC4>
+__global__ void __launch_bounds__(kAbsmaxThreads)
+absmax_kernel(const float* __restrict__ x, int64_t k, int64_t ldx, int64_t chunks_per_row,
+              int per_row, float* __restrict__ out) {
+    const int64_t row = blockIdx.x / chunks_per_row;
+    const int64_t e0 = (blockIdx.x % chunks_per_row) * kAbsmaxChunk;
+    const float* xr = x + row * ldx;
+    const int64_t e1 = min(e0 + (int64_t)kAbsmaxChunk, k);
+    float m = 0.0f;
+    if (VEC4) {
+        // row starts are 16-byte aligned and the chunk start is a multiple of 4 elements
+        const int64_t nvec = (e1 - e0) / 4;
+        const float4* xv = reinterpret_cast<const float4*>(xr + e0);
+#pragma unroll 8
+        for (int64_t i = threadIdx.x; i < nvec; i += kAbsmaxThreads) {
+            float4 v = __ldg(xv + i);
+            if (ACT == MPQ_ACT_HRELU) {
+                m = fmaxf(m, fmaxf(fmaxf(v.x, v.y), fmaxf(v.z, v.w)));
+            } else {
+                m = fmaxf(m, fmaxf(fmaxf(fabsf(v.x), fabsf(v.y)), fmaxf(fabsf(v.z), fabsf(v.w))));
+            }
+        }
+        for (int64_t i = e0 + nvec * 4 + threadIdx.x; i < e1; i += kAbsmaxThreads) {
+            float v = __ldg(xr + i);
+            m = fmaxf(m, ACT == MPQ_ACT_HRELU ? v : fabsf(v));
+        }
+    } else {
+        for (int64_t i = e0 + threadIdx.x; i < e1; i += kAbsmaxThreads) {
+            float v = __ldg(xr + i);
+            m = fmaxf(m, ACT == MPQ_ACT_HRELU ? v : fabsf(v));
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+    __shared__ float warp_max[kAbsmaxThreads / 32];
+    if ((threadIdx.x & 31) == 0) warp_max[threadIdx.x >> 5] = m;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+#pragma unroll
+        for (int w = 1; w < kAbsmaxThreads / 32; ++w) m = fmaxf(m, warp_max[w]);
+        if (m > 0.0f) atomicMax(reinterpret_cast<int*>(out + (per_row ? row : 0)), __float_as_int(m));
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// Row-major encoder.  One warp packs 1024 consecutive elements of a row (32 words per plane):
+// in step j lane L quantizes element 32 j + L (a fully coalesced 128-byte read), one
+// __ballot_sync per plane transposes that bit across the warp into word j, and lane j keeps it,
+// so the final store of each plane is again one coalesced 128-byte write.
+// ------------------------------------------------------------------------------------------
+constexpr int kEncodeThreads = 256;
+
+template <int BITS, int ACT>
+__global__ void __launch_bounds__(kEncodeThreads)
+encode_rows_kernel(const float* __restrict__ x, int64_t rows, int64_t k, int64_t ldx,
+                   const float* __restrict__ scale, int per_row,
+                   uint32_t* __restrict__ planes, int64_t rw, int64_t segs_per_row) {
+    const int64_t warp = (int64_t)blockIdx.x * (kEncodeThreads / 32) + (threadIdx.x >> 5);
+    if (warp >= rows * segs_per_row) return;
+    const int lane = threadIdx.x & 31;
+    const int64_t row = warp / segs_per_row;
+    const int64_t seg = warp % segs_per_row;
+    const float* xr = x + row * ldx;
+    const int64_t e0 = seg * 1024;
+
+    constexpr int H = 1 << (BITS - 1);
+    const float half_L = 0.5f * (float)((1 << BITS) - 1);
+    const float lo = (float)(-H), hi = (float)H - 0.5f;
+    const float inv = inverse_scale(__ldg(scale + (per_row ? row : 0)));
+
+    uint32_t mine[BITS];
+#pragma unroll
+    for (int p = 0; p < BITS; ++p) mine[p] = 0u;
+
+    const int64_t remaining = k - e0;                       // > 0 only for words that hold data
+    const int steps = remaining >= 1024 ? 32 : (int)((remaining + 31) / 32);   // warp-uniform
+    for (int j0 = 0; j0 < steps; j0 += 8) {
+        float v[8];
+        bool ok[8];
+#pragma unroll
+        for (int jj = 0; jj < 8; ++jj) {
+            const int64_t idx = e0 + (int64_t)(j0 + jj) * 32 + lane;
+            ok[jj] = idx < k;
+            v[jj] = ok[jj] ? __ldg(xr + idx) : 0.0f;
+        }
+#pragma unroll
+        for (int jj = 0; jj < 8; ++jj) {
+            const int u = ok[jj] ? level_index<ACT>(v[jj], inv, half_L, lo, hi, H) : 0;
+#pragma unroll
+            for (int p = 0; p < BITS; ++p) {
+                const uint32_t word = __ballot_sync(0xffffffffu, (u >> p) & 1);
+                if (lane == j0 + jj) mine[p] = word;
+            }
+        }
+    }
+    const int64_t word_idx = seg * 32 + lane;
+    if (word_idx < rw) {
+#pragma unroll
+        for (int p = 0; p < BITS; ++p) planes[((int64_t)p * rows + row) * rw + word_idx] = mine[p];
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// NCHW activations -> planes[bits][N][H][W][C/32].  A warp takes 32 pixels x 32 channels:
+// lane = pixel, so each of the 32 channel reads is a coalesced 128-byte row of one channel,
+// and every lane builds the word of its own pixel bit by bit (channel c -> bit c).
+// ------------------------------------------------------------------------------------------
+template <int BITS, int ACT>
+__global__ void __launch_bounds__(kEncodeThreads)
+encode_nchw_kernel(const float* __restrict__ x, int N, int C, int64_t HW,
+                   const float* __restrict__ scale, uint32_t* __restrict__ planes,
+                   int64_t pix_blocks, int64_t total_warps) {
+    const int64_t warp = (int64_t)blockIdx.x * (kEncodeThreads / 32) + (threadIdx.x >> 5);
+    if (warp >= total_warps) return;
+    const int lane = threadIdx.x & 31;
+    const int Cw = C / 32;
+    const int64_t pb = warp % pix_blocks;
+    const int64_t rest = warp / pix_blocks;
+    const int cw = (int)(rest % Cw);
+    const int64_t n = rest / Cw;
+    const int64_t pixel = pb * 32 + lane;
+    const bool valid = pixel < HW;
+
+    constexpr int H = 1 << (BITS - 1);
+    const float half_L = 0.5f * (float)((1 << BITS) - 1);
+    const float lo = (float)(-H), hi = (float)H - 0.5f;
+    const float inv = inverse_scale(__ldg(scale));
+
+    const float* base = x + ((n * C + (int64_t)cw * 32) * HW + pixel);
+    uint32_t word[BITS];
+#pragma unroll
+    for (int p = 0; p < BITS; ++p) word[p] = 0u;
+#pragma unroll
+    for (int c0 = 0; c0 < 32; c0 += 8) {
+        float v[8];
+#pragma unroll
+        for (int cc = 0; cc < 8; ++cc) v[cc] = valid ? __ldg(base + (int64_t)(c0 + cc) * HW) : 0.0f;
+#pragma unroll
+        for (int cc = 0; cc < 8; ++cc) {
+            const uint32_t u = (uint32_t)level_index<ACT>(v[cc], inv, half_L, lo, hi, H);
+#pragma unroll
+            for (int p = 0; p < BITS; ++p) word[p] |= ((u >> p) & 1u) << (c0 + cc);
+        }
+    }
+    if (valid) {
+#pragma unroll
+        for (int p = 0; p < BITS; ++p)
+            planes[(((int64_t)p * N + n) * HW + pixel) * Cw + cw] = word[p];
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// OIHW weights -> planes[bits][O][row_words(KH*KW*C)], k ordered (kh, kw, c); plus tap sums.
+// Weights are encoded once, offline: one thread per output word, no tuning.
+// ------------------------------------------------------------------------------------------
+template <int ACT>
+__device__ __forceinline__ int level_index_rt(float x, float inv, int bits) {
+    const int H = 1 << (bits - 1);
+    return level_index<ACT>(x, inv, 0.5f * (float)((1 << bits) - 1), (float)(-H), (float)H - 0.5f, H);
+}
+
+__global__ void encode_oihw_kernel(const float* __restrict__ w, int O, int C, int taps,
+                                   const float* __restrict__ scale, int per_row, int bits,
+                                   uint32_t* __restrict__ planes, int64_t rw) {
+    const int64_t id = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (id >= (int64_t)O * rw) return;
+    const int64_t o = id / rw;
+    const int64_t word = id % rw;
+    const int64_t K = (int64_t)taps * C;
+    const float inv = inverse_scale(__ldg(scale + (per_row ? o : 0)));
+    uint32_t out[kMaxBits];
+    for (int p = 0; p < kMaxBits; ++p) out[p] = 0u;
+    for (int t = 0; t < 32; ++t) {
+        const int64_t kidx = word * 32 + t;
+        if (kidx >= K) break;
+        const int64_t tap = kidx / C, c = kidx % C;
+        const uint32_t u = (uint32_t)level_index_rt<MPQ_ACT_HTANH>(__ldg(w + (o * C + c) * taps + tap), inv, bits);
+        for (int p = 0; p < kMaxBits; ++p) out[p] |= ((u >> p) & 1u) << t;
+    }
+    for (int p = 0; p < bits; ++p) planes[((int64_t)p * O + o) * rw + word] = out[p];
+}
+
+__global__ void tap_sums_kernel(const float* __restrict__ w, int O, int C, int taps,
+                                const float* __restrict__ scale, int per_row, int bits,
+                                int32_t* __restrict__ tap_sums) {
+    const int64_t id = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (id >= (int64_t)O * taps) return;
+    const int64_t tap = id / O, o = id % O;
+    const float inv = inverse_scale(__ldg(scale + (per_row ? o : 0)));
+    const int L = (1 << bits) - 1;
+    int32_t s = 0;
+    for (int c = 0; c < C; ++c)
+        s += 2 * level_index_rt<MPQ_ACT_HTANH>(__ldg(w + (o * C + c) * taps + tap), inv, bits) - L;
+    tap_sums[tap * O + o] = s;
+}
+
+__global__ void add_relu_kernel(const float* __restrict__ a, const float* __restrict__ b,
+                                float* __restrict__ y, int64_t n) {
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride) {
+        const float v = b ? __fadd_rn(a[i], b[i]) : a[i];
+        y[i] = fmaxf(v, 0.0f);
+    }
+}
+
+template <template <int, int> class Launcher, typename... Args>
+static int dispatch_bits_act(int bits, int act, Args... args) {
+#define MPQ_CASE(B)                                                              \
+    case B:                                                                      \
+        return act == MPQ_ACT_HRELU ? Launcher<B, MPQ_ACT_HRELU>::run(args...)   \
+                                    : Launcher<B, MPQ_ACT_HTANH>::run(args...);
+    switch (bits) {
+        MPQ_CASE(1) MPQ_CASE(2) MPQ_CASE(3) MPQ_CASE(4) MPQ_CASE(5) MPQ_CASE(6) MPQ_CASE(7) MPQ_CASE(8)
+    }
+#undef MPQ_CASE
+    return MPQ_ERR_UNSUPPORTED;
+}
+
+template <int BITS, int ACT>
+struct EncodeRowsLauncher {
+    static int run(const float* x, int64_t rows, int64_t k, int64_t ldx, const float* scale, int per_row,
+                   uint32_t* planes, cudaStream_t st) {
+        const int64_t rw = row_words(k);
+        const int64_t segs = ceil_div(rw, 32);
+        const int64_t warps = rows * segs;
+        const int64_t blocks = ceil_div(warps, kEncodeThreads / 32);
+        if (blocks > 0x7fffffffLL) return MPQ_ERR_BAD_SHAPE;
+        encode_rows_kernel<BITS, ACT><<<(unsigned)blocks, kEncodeThreads, 0, st>>>(
+            x, rows, k, ldx, scale, per_row, planes, rw, segs);
+        return launch_status();
+    }
+};
+
+template <int BITS, int ACT>
+struct EncodeNchwLauncher {
+    static int run(const float* x, int N, int C, int64_t HW, const float* scale, uint32_t* planes, cudaStream_t st) {
+        const int64_t pix_blocks = ceil_div(HW, 32);
+        const int64_t warps = pix_blocks * (C / 32) * N;
+        const int64_t blocks = ceil_div(warps, kEncodeThreads / 32);
+        if (blocks > 0x7fffffffLL) return MPQ_ERR_BAD_SHAPE;
+        encode_nchw_kernel<BITS, ACT><<<(unsigned)blocks, kEncodeThreads, 0, st>>>(
+            x, N, C, HW, scale, planes, pix_blocks, warps);
+        return launch_status();
+    }
+};
+
+}  // namespace mpq
+
+using namespace mpq;
+
+extern "C" int mpq_absmax(const float* x, int64_t rows, int64_t k, int64_t ldx, int mode, int act,
+                          float* scale_out, void* stream) {
+    if (!x || !scale_out) return MPQ_ERR_NULL;
+    if (rows <= 0 || k <= 0 || ldx < k) return MPQ_ERR_BAD_SHAPE;
+    if ((mode != MPQ_SCALE_PER_TENSOR && mode != MPQ_SCALE_PER_ROW) ||
+        (act != MPQ_ACT_HTANH && act != MPQ_ACT_HRELU)) return MPQ_ERR_UNSUPPORTED;
+    cudaStream_t st = (cudaStream_t)stream;
+    const int per_row = mode == MPQ_SCALE_PER_ROW;
+    if (cudaMemsetAsync(scale_out, 0, sizeof(float) * (per_row ? rows : 1), st) != cudaSuccess) return MPQ_ERR_CUDA;
+    if (!per_row && ldx == k) { k = rows * k; ldx = k; rows = 1; }   // contiguous tensor: one long row
+    const int64_t chunks = ceil_div(k, kAbsmaxChunk);
+    const int64_t blocks = rows * chunks;
+    if (blocks > 0x7fffffffLL) return MPQ_ERR_BAD_SHAPE;
+    const bool vec4 = aligned16(x) && (ldx % 4 == 0);
+#define MPQ_LAUNCH(A, V) absmax_kernel<A, V><<<(unsigned)blocks, kAbsmaxThreads, 0, st>>>(x, k, ldx, chunks, per_row, scale_out)
+    if (act == MPQ_ACT_HRELU) { if (vec4) MPQ_LAUNCH(MPQ_ACT_HRELU, true); else MPQ_LAUNCH(MPQ_ACT_HRELU, false); }
+    else                      { if (vec4) MPQ_LAUNCH(MPQ_ACT_HTANH, true); else MPQ_LAUNCH(MPQ_ACT_HTANH, false); }
+#undef MPQ_LAUNCH
+    return launch_status();
+}
+
+extern "C" int mpq_encode(const float* x, int64_t rows, int64_t k, int64_t ldx,
+                          const float* scale, int mode, int act, int bits,
+                          uint32_t* planes, void* stream) {
+    if (!x || !scale || !planes) return MPQ_ERR_NULL;
+    if (rows <= 0 || k <= 0 || ldx < k) return MPQ_ERR_BAD_SHAPE;
+    if (!bits_ok(bits) || (mode != MPQ_SCALE_PER_TENSOR && mode != MPQ_SCALE_PER_ROW) ||
+        (act != MPQ_ACT_HTANH && act != MPQ_ACT_HRELU)) return MPQ_ERR_UNSUPPORTED;
+    if (!aligned16(planes)) return MPQ_ERR_ALIGN;
+    return dispatch_bits_act<EncodeRowsLauncher>(bits, act, x, rows, k, ldx, scale,
+                                                 (int)(mode == MPQ_SCALE_PER_ROW), planes, (cudaStream_t)stream);
+}
+
+static bool conv_channels_ok(int C) { return C == 32 || C == 64 || (C > 0 && C % 128 == 0); }
+
+extern "C" int mpq_encode_nchw(const float* x, int N, int C, int H, int W, const float* scale, int act,
+                               int bits, uint32_t* planes, void* stream) {
+    if (!x || !scale || !planes) return MPQ_ERR_NULL;
+    if (N <= 0 || C <= 0 || H <= 0 || W <= 0) return MPQ_ERR_BAD_SHAPE;
+    if (!bits_ok(bits) || !conv_channels_ok(C) || (act != MPQ_ACT_HTANH && act != MPQ_ACT_HRELU)) return MPQ_ERR_UNSUPPORTED;
+    if (!aligned16(planes)) return MPQ_ERR_ALIGN;
+    return dispatch_bits_act<EncodeNchwLauncher>(bits, act, x, N, C, (int64_t)H * W, scale, planes, (cudaStream_t)stream);
+}
+
+extern "C" int mpq_encode_oihw(const float* w, int O, int C, int KH, int KW, const float* scale, int mode,
+                               int bits, uint32_t* planes, int32_t* tap_sums, void* stream) {
+    if (!w || !scale || !planes || !tap_sums) return MPQ_ERR_NULL;
+    if (O <= 0 || C <= 0 || KH <= 0 || KW <= 0) return MPQ_ERR_BAD_SHAPE;
+    if (!bits_ok(bits) || !conv_channels_ok(C) || (mode != MPQ_SCALE_PER_TENSOR && mode != MPQ_SCALE_PER_ROW)) return MPQ_ERR_UNSUPPORTED;
+    if (!aligned16(planes)) return MPQ_ERR_ALIGN;
+    cudaStream_t st = (cudaStream_t)stream;
+    const int taps = KH * KW;
+    const int64_t rw = row_words((int64_t)taps * C);
+    const int per_row = mode == MPQ_SCALE_PER_ROW;
+    encode_oihw_kernel<<<(unsigned)ceil_div((int64_t)O * rw, 128), 128, 0, st>>>(w, O, C, taps, scale, per_row, bits, planes, rw);
+    if (launch_status() != MPQ_OK) return MPQ_ERR_CUDA;
+    tap_sums_kernel<<<(unsigned)ceil_div((int64_t)O * taps, 128), 128, 0, st>>>(w, O, C, taps, scale, per_row, bits, tap_sums);
+    return launch_status();
+}
+
+extern "C" int mpq_add_relu(const float* a, const float* b, float* y, int64_t n, void* stream) {
+    if (!a || !y) return MPQ_ERR_NULL;
+    if (n <= 0) return MPQ_ERR_BAD_SHAPE;
+    const int64_t blocks = min((int64_t)148 * 16, ceil_div(n, 256));
+    add_relu_kernel<<<(unsigned)blocks, 256, 0, (cudaStream_t)stream>>>(a, b, y, n);
+    return launch_status();
+}

@@ -1,0 +1,97 @@
+// C-ABI entry points of the layer product: argument checks, then dispatch on the bit-widths.
+#include "mpq_branch_kernel.cuh"
+
+namespace mpq {
+
+template <int HB> int launch_gemm_hb(int sb, const BranchParams& p, cudaStream_t st);
+template <int HB> int launch_conv_hb(int sb, const BranchParams& p, cudaStream_t st);
+
+static int dispatch_gemm(int hb, int sb, const BranchParams& p, cudaStream_t st) {
+    switch (hb) {
+        case 1: return launch_gemm_hb<1>(sb, p, st);
+        case 2: return launch_gemm_hb<2>(sb, p, st);
+        case 3: return launch_gemm_hb<3>(sb, p, st);
+        case 4: return launch_gemm_hb<4>(sb, p, st);
+        case 5: return launch_gemm_hb<5>(sb, p, st);
+        case 6: return launch_gemm_hb<6>(sb, p, st);
+        case 7: return launch_gemm_hb<7>(sb, p, st);
+        case 8: return launch_gemm_hb<8>(sb, p, st);
+    }
+    return MPQ_ERR_UNSUPPORTED;
+}
+
+static int dispatch_conv(int hb, int sb, const BranchParams& p, cudaStream_t st) {
+    switch (hb) {
+        case 1: return launch_conv_hb<1>(sb, p, st);
+        case 2: return launch_conv_hb<2>(sb, p, st);
+        case 3: return launch_conv_hb<3>(sb, p, st);
+        case 4: return launch_conv_hb<4>(sb, p, st);
+        case 5: return launch_conv_hb<5>(sb, p, st);
+        case 6: return launch_conv_hb<6>(sb, p, st);
+        case 7: return launch_conv_hb<7>(sb, p, st);
+        case 8: return launch_conv_hb<8>(sb, p, st);
+    }
+    return MPQ_ERR_UNSUPPORTED;
+}
+
+// k * L_a * L_w must stay below 2^31 so that every |acc| fits int32.
+static bool int32_headroom(int64_t k, int a_bits, int w_bits) {
+    const int64_t LL = (int64_t)((1 << a_bits) - 1) * ((1 << w_bits) - 1);
+    return k < ((int64_t)1 << 31) && k * LL < ((int64_t)1 << 31);
+}
+
+}  // namespace mpq
+
+using namespace mpq;
+
+extern "C" int mpq_gemm(const uint32_t* a_planes, int a_bits, const uint32_t* b_planes, int b_bits,
+                        int64_t m, int64_t n, int64_t k,
+                        int32_t* c_i32, float* c_f32, int64_t ldc,
+                        const float* a_scale, const float* b_scale, int b_mode, void* stream) {
+    if (!a_planes || !b_planes || (!c_i32 && !c_f32)) return MPQ_ERR_NULL;
+    if (c_f32 && (!a_scale || !b_scale)) return MPQ_ERR_NULL;
+    if (m <= 0 || n <= 0 || k <= 0 || ldc < n) return MPQ_ERR_BAD_SHAPE;
+    if (!bits_ok(a_bits) || !bits_ok(b_bits) ||
+        (b_mode != MPQ_SCALE_PER_TENSOR && b_mode != MPQ_SCALE_PER_ROW)) return MPQ_ERR_UNSUPPORTED;
+    if (!int32_headroom(k, a_bits, b_bits)) return MPQ_ERR_OVERFLOW;
+    if (!aligned16(a_planes) || !aligned16(b_planes)) return MPQ_ERR_ALIGN;
+    BranchParams p = {};
+    p.held = a_planes; p.streamed = b_planes;
+    p.held_rows = m; p.streamed_rows = n;
+    p.rw = row_words(k); p.k = k;
+    p.out_i32 = c_i32; p.out_f32 = c_f32; p.ldc = ldc;
+    p.a_scale = a_scale; p.w_scale = b_scale; p.w_per_row = b_mode == MPQ_SCALE_PER_ROW;
+    return dispatch_gemm(a_bits, b_bits, p, (cudaStream_t)stream);
+}
+
+extern "C" int mpq_conv(const uint32_t* x_planes, int a_bits, int N, int C, int H, int W,
+                        const uint32_t* w_planes, int w_bits, const int32_t* tap_sums,
+                        int O, int KH, int KW, int stride, int pad,
+                        int32_t* y_i32, float* y_f32,
+                        const float* x_scale, const float* w_scale, int w_mode, void* stream) {
+    if (!x_planes || !w_planes || (!y_i32 && !y_f32)) return MPQ_ERR_NULL;
+    if (y_f32 && (!x_scale || !w_scale)) return MPQ_ERR_NULL;
+    if (N <= 0 || C <= 0 || H <= 0 || W <= 0 || O <= 0) return MPQ_ERR_BAD_SHAPE;
+    if (!bits_ok(a_bits) || !bits_ok(w_bits) || !((KH == 1 && KW == 1) || (KH == 3 && KW == 3)) ||
+        (stride != 1 && stride != 2) || pad < 0 || pad > 1 ||
+        !(C == 32 || C == 64 || C % 128 == 0) ||
+        (w_mode != MPQ_SCALE_PER_TENSOR && w_mode != MPQ_SCALE_PER_ROW)) return MPQ_ERR_UNSUPPORTED;
+    if (pad > 0 && !tap_sums) return MPQ_ERR_NULL;
+    if (H + 2 * pad < KH || W + 2 * pad < KW) return MPQ_ERR_BAD_SHAPE;
+    const int64_t K = (int64_t)KH * KW * C;
+    if (!int32_headroom(K, a_bits, w_bits)) return MPQ_ERR_OVERFLOW;
+    if (!aligned16(x_planes) || !aligned16(w_planes)) return MPQ_ERR_ALIGN;
+    BranchParams p = {};
+    p.held = w_planes; p.streamed = x_planes;
+    p.Ho = (H + 2 * pad - KH) / stride + 1;
+    p.Wo = (W + 2 * pad - KW) / stride + 1;
+    p.held_rows = O; p.streamed_rows = (int64_t)N * p.Ho * p.Wo;
+    p.rw = row_words(K); p.k = K;
+    p.out_i32 = y_i32; p.out_f32 = y_f32; p.ldc = 0;
+    p.a_scale = x_scale; p.w_scale = w_scale; p.w_per_row = w_mode == MPQ_SCALE_PER_ROW;
+    p.N = N; p.C = C; p.H = H; p.W = W; p.O = O; p.KH = KH; p.KW = KW; p.stride = stride; p.pad = pad;
+    p.Cw = C / 32; p.granule = p.Cw >= 4 ? 4 : p.Cw;
+    p.tap_sums = tap_sums;
+    // held = weights (w_bits planes), streamed = activations (a_bits planes)
+    return dispatch_conv(w_bits, a_bits, p, (cudaStream_t)stream);
+}

@@ -15,3 +15,22 @@ def pytest_configure(config):
 @pytest.fixture(scope="session")
 def golden_dir():
     return os.path.join(ROOT, "tests", "golden")
+
+
+@pytest.fixture(scope="session")
+def mpq():
+    """The Python binding over libmpq.so, built in-tree on demand (nvcc cross-compiles without a GPU)."""
+    from paper_1905_13389_b200 import binding, build
+    if not os.path.exists(binding.LIB_PATH):
+        build.build()
+    binding.lib()
+    return binding
+
+
+@pytest.fixture(scope="session")
+def cuda(mpq):
+    import torch
+    if not torch.cuda.is_available():
+        pytest.fail("GPU tests need a CUDA device; run them with -m gpu on a B200")
+    torch.cuda.set_device(0)
+    return torch.device("cuda:0")
