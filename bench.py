@@ -1,0 +1,310 @@
+#!/usr/bin/env python
+"""Benchmark of the encoded-layer hot path on B200.
+
+One step = one pass of the whole path over one batch of synthetic input, through the C ABI:
+range (max-abs) of both operands -> fused quantize+pack of both -> branch-fused binary GEMM with
+the decoder scale fused into the store (int32 accumulators and scaled fp32 output).
+Workload at N = 1: the W2A2 square GEMM m = n = k = 4096 of the bit-width sweep (the setting the
+throughput target is quoted on).  With N > 1 every rank runs the same workload on its own GPU
+(independent problems, no exchange step): weak scaling, replicas only.
+
+Prints ONE JSON line (rank 0).  ``--impl reference`` times the CPU oracle instead.
+``--full FILE`` additionally writes per-workload numbers (sweep, FC, conv, encoders) to FILE.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "equivalent W2A2 TOPS of the encoded layer (2*m*n*k / step time)"
+UNIT = "TOPS"
+SIZE = 4096
+A_BITS = W_BITS = 2
+HBM_FALLBACK_GBS = 6650.0      # used only when MEASURED_PEAKS.json is absent
+# DRAM bytes per launch of the GEMM kernel from the committed ncu capture
+# (profiles/branch_kernel_w2a2_4096.md); None until a capture exists.
+GEMM_DRAM_TRAFFIC_BYTES = None
+
+
+def _peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return json.load(f), "measured"
+    return {"hbm_gbs": HBM_FALLBACK_GBS}, "fallback"
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons every 200 ms while the timed region runs."""
+    QUERY = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+             "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.rows = []
+        self.proc = None
+
+    def __enter__(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.QUERY, "--format=csv,noheader,nounits",
+                 "-lms", "200"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+        return self
+
+    def _read(self):
+        for line in self.proc.stdout:
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) >= 7:
+                self.rows.append(parts)
+
+    def __exit__(self, *exc):
+        if self.proc is not None:
+            time.sleep(0.25)
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except subprocess.TimeoutExpired:
+                self.proc.kill()
+
+    def summary(self):
+        sm, mx, reasons = [], [], set()
+        for r in self.rows:
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1]))
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def _workload_arrays():
+    from paper_1905_13389_b200 import inputs
+    c = inputs.config4(W_BITS, A_BITS, SIZE)
+    return c["x"], c["w"]
+
+
+# ------------------------------------------------------------------------------------------------
+# reference arm / cpu_baseline: the oracle as it stands, on the host cores, on a bounded sample
+# ------------------------------------------------------------------------------------------------
+def _oracle_sample_step(x, w, rows):
+    """Oracle pass over `rows` rows of the activations against the full weight matrix."""
+    import oracle
+    s_a = oracle.absmax(x)
+    s_w = oracle.absmax(w)
+    qa = oracle.quantize(x[:rows], s_a, A_BITS)
+    qb = oracle.quantize(w, s_w, W_BITS)
+    acc = oracle.gemm(qa, qb)
+    return oracle.scale(acc, s_a[0], s_w, A_BITS, W_BITS)
+
+
+def _time_oracle(x, w, rows, steps, warmup):
+    import oracle
+    oracle.build()
+    for _ in range(warmup):
+        _oracle_sample_step(x, w, rows)
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        _oracle_sample_step(x, w, rows)
+    dt = (time.perf_counter() - t0) / steps
+    tops = 2.0 * rows * SIZE * SIZE / dt / 1e12
+    sample = "rows 0..%d of the %dx%d activations against all %d weight rows (k=%d): range, quantize, " \
+             "integer GEMM and scale; throughput = 2*rows*n*k / time" % (rows - 1, SIZE, SIZE, SIZE, SIZE)
+    return tops, dt, oracle.threads(), sample
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    x, w = _workload_arrays()
+    rows = 1024
+    tops, dt, cores, sample = _time_oracle(x, w, rows, args.steps, min(args.warmup, 1))
+    line = {
+        "impl": "reference", "metric": METRIC, "value": tops, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": min(args.warmup, 1), "ms_per_step": dt * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "int32", "data": "synthetic",
+        "config": {"workload": "gemm_w2a2_4096 (bounded sample: %d rows per step)" % rows, "m": SIZE, "n": SIZE, "k": SIZE,
+                   "a_bits": A_BITS, "w_bits": W_BITS},
+        "cpu_baseline": {"value": tops, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": tops, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ------------------------------------------------------------------------------------------------
+# CUDA arm
+# ------------------------------------------------------------------------------------------------
+def run_cuda(args):
+    import torch
+    import torch.distributed as dist
+    from paper_1905_13389_b200 import binding as mpq
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    mpq.lib()
+
+    x_np, w_np = _workload_arrays()
+    x = torch.from_numpy(x_np).to(dev)
+    w = torch.from_numpy(w_np).to(dev)
+    m = n = k = SIZE
+    rw = mpq.row_words(k)
+    s_a = torch.empty(1, dtype=torch.float32, device=dev)
+    s_w = torch.empty(1, dtype=torch.float32, device=dev)
+    ap = torch.empty((A_BITS, m, rw), dtype=torch.int32, device=dev)
+    wp = torch.empty((W_BITS, n, rw), dtype=torch.int32, device=dev)
+    ci = torch.empty((m, n), dtype=torch.int32, device=dev)
+    cf = torch.empty((m, n), dtype=torch.float32, device=dev)
+
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    enc_events, gemm_events = [], []
+
+    def step(record: bool):
+        mpq.absmax(x, mpq.SCALE_PER_TENSOR, mpq.ACT_HTANH, out=s_a)
+        mpq.absmax(w, mpq.SCALE_PER_TENSOR, mpq.ACT_HTANH, out=s_w)
+        if record:
+            e0, e1, e2 = ev(), ev(), ev()
+            e0.record()
+        mpq.encode(x, s_a, A_BITS, out=ap)
+        mpq.encode(w, s_w, W_BITS, out=wp)
+        if record:
+            e1.record()
+        mpq.gemm(ap, A_BITS, wp, W_BITS, m, n, k, ci, cf, s_a, s_w, mpq.SCALE_PER_TENSOR)
+        if record:
+            e2.record()
+            enc_events.append((e0, e1))
+            gemm_events.append((e1, e2))
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        step(False)
+    barrier()
+    popc_peak, probe_mhz, sms = mpq.measure_popc_peak()     # roofline denominator, measured live
+
+    with ClockSampler(local_rank) as clocks:
+        barrier()
+        t0, t1 = ev(), ev()
+        t0.record()
+        for _ in range(args.steps):
+            step(True)
+        t1.record()
+        barrier()
+    elapsed_ms = t0.elapsed_time(t1)
+    if world > 1:
+        t = torch.tensor([elapsed_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        elapsed_ms = float(t.item())
+    ms_per_step = elapsed_ms / args.steps
+    value = world * 2.0 * m * n * k / (ms_per_step * 1e-3) / 1e12
+
+    gemm_ms = statistics.mean(a.elapsed_time(b) for a, b in gemm_events)
+    enc_ms = statistics.mean(a.elapsed_time(b) for a, b in enc_events)
+    popcs = float(A_BITS * W_BITS) * m * n * (k // 32)                 # algorithmic popcounts per launch
+    achieved = popcs / (gemm_ms * 1e-3)
+    peaks, peak_kind = _peaks()
+    enc_bytes = (m * k + n * k) * 4.0 + (A_BITS * m + W_BITS * n) * rw * 4.0
+    enc_gbs = enc_bytes / (enc_ms * 1e-3) / 1e9
+
+    # end to end through the host-buffer entry point: pinned host inputs, H2D + D2H inside the timed region
+    xh, wh = torch.from_numpy(x_np).pin_memory(), torch.from_numpy(w_np).pin_memory()
+    oi = torch.empty((m, n), dtype=torch.int32).pin_memory()
+    of = torch.empty((m, n), dtype=torch.float32).pin_memory()
+    ws = torch.empty(mpq.linear_host_workspace(m, n, k, A_BITS, W_BITS), dtype=torch.uint8, device=dev)
+    e2e_steps = max(3, min(args.steps, 10))
+    for _ in range(2):
+        mpq.linear_host(xh, wh, A_BITS, W_BITS, out_i32_host=oi, out_f32_host=of, workspace=ws)
+    barrier()
+    t0, t1 = ev(), ev()
+    t0.record()
+    for _ in range(e2e_steps):
+        mpq.linear_host(xh, wh, A_BITS, W_BITS, out_i32_host=oi, out_f32_host=of, workspace=ws)
+    t1.record()
+    barrier()
+    e2e_ms = t0.elapsed_time(t1)
+    if world > 1:
+        t = torch.tensor([e2e_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+    e2e_value = world * 2.0 * m * n * k / (e2e_ms / e2e_steps * 1e-3) / 1e12
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "int32", "data": "synthetic",
+            "config": {"workload": "gemm_w2a2_4096", "m": m, "n": n, "k": k, "a_bits": A_BITS, "w_bits": W_BITS,
+                       "step": "absmax x2 + encode x2 + branch-fused GEMM (int32 + scaled fp32 out)",
+                       "l2": "fp32 inputs (128 MiB) and outputs (128 MiB) per step exceed the 126 MB L2; no flush",
+                       "binary_tops": value * A_BITS * W_BITS},
+            "roofline": {"bound": "alu", "kernel": "branch_kernel<2,2> (XOR+POPC GEMM)",
+                         "achieved": achieved / 1e9, "peak": popc_peak / 1e9, "unit": "Gpopc/s",
+                         "frac": achieved / popc_peak, "traffic": GEMM_DRAM_TRAFFIC_BYTES,
+                         "peak_source": "POPC issue rate measured live by mpq_measure_popc_peak at %.0f MHz on %d SMs "
+                                        "(%.1f lanes/clk/SM)" % (probe_mhz, sms, popc_peak / (probe_mhz * 1e6 * sms)),
+                         "ms_per_launch": gemm_ms, "algorithmic_popc_per_launch": popcs},
+            "encode": {"bound": "hbm", "achieved": enc_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                       "frac": enc_gbs / peaks["hbm_gbs"], "peak_source": "%s copy bandwidth" % peak_kind,
+                       "ms_per_step": enc_ms, "bytes_per_step": enc_bytes},
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": 2 * m * k * 4,
+                    "d2h_bytes_per_step": 2 * m * n * 4, "ms_per_step": e2e_ms / e2e_steps,
+                    "api": "mpq_linear_host (pinned host buffers)"},
+            "gpu_launches": 5 * args.steps,
+            "clocks": clocks.summary(),
+        }
+        if world == 1 and not args.no_cpu_baseline:
+            tops, dt, cores, sample = _time_oracle(x_np, w_np, 1024, 4, 1)
+            line["cpu_baseline"] = {"value": tops, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample,
+                                    "seconds_per_sample": dt}
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_cuda(args)
+
+
+if __name__ == "__main__":
+    main()
