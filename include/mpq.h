@@ -12,7 +12,7 @@
  * Conventions for every entry point
  *   - Pointers are DEVICE pointers unless the name ends in _host.  The caller owns and
  *     sizes every buffer; the library allocates nothing and keeps no state between calls
- *     (exception: mpq_linear_host stages through a caller-provided device workspace).
+ *     (mpq_linear and mpq_linear_host stage through a caller-provided device workspace).
  *   - Calls are asynchronous on `stream` (a cudaStream_t passed as void*; NULL = the
  *     default stream) unless stated otherwise.  Outputs are fully overwritten.
  *   - Return value: an mpq_status.  Errors that the host can see (null pointers, bad
@@ -122,12 +122,23 @@ int mpq_conv(const uint32_t* x_planes, int a_bits, int N, int C, int H, int W,
  * b may be NULL (plain ReLU).  n elements, fp32, one rounded add. */
 int mpq_add_relu(const float* a, const float* b, float* y, int64_t n, void* stream);
 
-/* ---- Whole encoded fully-connected layer from HOST buffers (Fig. 1 end to end):
- * copies x_host [m x k] and w_host [n x k] to the device workspace, takes both ranges
- * (activations per tensor with `a_act`, weights per `w_mode`), encodes both, runs mpq_gemm,
- * and copies out_i32_host / out_f32_host [m x n] back (either may be NULL, not both).
- * Host buffers should be pinned for the copies to be asynchronous.  The call returns after
- * the stream has drained (it synchronizes `stream`).
+/* ---- Whole encoded fully-connected layer (Fig. 1 end to end: Encoder of both operands,
+ * the a_bits x w_bits branches, Decoder): out = decode(encode(x) . encode(w)^T).
+ * x [m x k] and w [n x k] are dense fp32 DEVICE tensors; activations take one range with `a_act`,
+ * weights one range (PER_TENSOR) or one per output row (PER_ROW).  out_i32 / out_f32 [m x n],
+ * dense; either may be NULL, not both.
+ * workspace: device memory of at least mpq_linear_workspace() bytes, 256-byte aligned, holding the
+ * two ranges and the two packed operands for the duration of the call (contents undefined after). */
+int64_t mpq_linear_workspace(int64_t m, int64_t n, int64_t k, int a_bits, int w_bits);
+int mpq_linear(const float* x, const float* w, int64_t m, int64_t n, int64_t k,
+               int a_bits, int w_bits, int a_act, int w_mode,
+               int32_t* out_i32, float* out_f32,
+               void* workspace, int64_t workspace_bytes, void* stream);
+
+/* The same layer from HOST buffers: copies x_host and w_host into the device workspace, runs
+ * mpq_linear there, and copies out_i32_host / out_f32_host [m x n] back (either may be NULL, not
+ * both).  Host buffers should be pinned for the copies to be asynchronous.  The call returns
+ * after the stream has drained (it synchronizes `stream`).
  * workspace: device memory of at least mpq_linear_host_workspace() bytes, 256-byte aligned. */
 int64_t mpq_linear_host_workspace(int64_t m, int64_t n, int64_t k, int a_bits, int w_bits);
 int mpq_linear_host(const float* x_host, const float* w_host, int64_t m, int64_t n, int64_t k,

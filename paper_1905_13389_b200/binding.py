@@ -52,13 +52,16 @@ def lib() -> ctypes.CDLL:
         L.mpq_gemm.argtypes = [P, i32, P, i32, i64, i64, i64, P, P, i64, P, P, i32, P]
         L.mpq_conv.argtypes = [P, i32, i32, i32, i32, i32, P, i32, P, i32, i32, i32, i32, i32, P, P, P, P, i32, P]
         L.mpq_add_relu.argtypes = [P, P, P, i64, P]
+        L.mpq_linear_workspace.argtypes = [i64, i64, i64, i32, i32]
+        L.mpq_linear_workspace.restype = i64
+        L.mpq_linear.argtypes = [P, P, i64, i64, i64, i32, i32, i32, i32, P, P, P, i64, P]
         L.mpq_linear_host_workspace.argtypes = [i64, i64, i64, i32, i32]
         L.mpq_linear_host_workspace.restype = i64
         L.mpq_linear_host.argtypes = [P, P, i64, i64, i64, i32, i32, i32, i32, P, P, P, i64, P]
         L.mpq_measure_popc_peak.argtypes = [ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double),
                                             ctypes.POINTER(ctypes.c_int), P]
         for name in ("mpq_absmax", "mpq_encode", "mpq_encode_nchw", "mpq_encode_oihw", "mpq_gemm", "mpq_conv",
-                     "mpq_add_relu", "mpq_linear_host", "mpq_measure_popc_peak"):
+                     "mpq_add_relu", "mpq_linear", "mpq_linear_host", "mpq_measure_popc_peak"):
             getattr(L, name).restype = i32
         _lib = L
     return _lib
@@ -174,6 +177,25 @@ def add_relu(a: torch.Tensor, b: Optional[torch.Tensor], y: torch.Tensor) -> tor
     _check(lib().mpq_add_relu(_ptr(a, torch.float32), _ptr(b, torch.float32), _ptr(y, torch.float32),
                               a.numel(), _stream()), "mpq_add_relu")
     return y
+
+
+def linear_workspace(m: int, n: int, k: int, a_bits: int, w_bits: int) -> int:
+    return int(lib().mpq_linear_workspace(m, n, k, a_bits, w_bits))
+
+
+def linear(x: torch.Tensor, w: torch.Tensor, a_bits: int, w_bits: int,
+           a_act: int = ACT_HTANH, w_mode: int = SCALE_PER_TENSOR,
+           out_i32: Optional[torch.Tensor] = None, out_f32: Optional[torch.Tensor] = None,
+           workspace: Optional[torch.Tensor] = None):
+    """Whole encoded fully-connected layer on device tensors: x [m x k], w [n x k] -> [m x n]."""
+    m, k = x.shape
+    n, _ = w.shape
+    if workspace is None:
+        workspace = torch.empty(linear_workspace(m, n, k, a_bits, w_bits), dtype=torch.uint8, device=x.device)
+    _check(lib().mpq_linear(_ptr(x, torch.float32), _ptr(w, torch.float32), m, n, k, a_bits, w_bits, a_act, w_mode,
+                            _ptr(out_i32, torch.int32), _ptr(out_f32, torch.float32),
+                            workspace.data_ptr(), workspace.numel(), _stream()), "mpq_linear")
+    return out_i32, out_f32
 
 
 def linear_host_workspace(m: int, n: int, k: int, a_bits: int, w_bits: int) -> int:

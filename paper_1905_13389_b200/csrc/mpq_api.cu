@@ -24,31 +24,87 @@ extern "C" int64_t mpq_packed_words(int64_t rows, int64_t k, int bits) {
     return (int64_t)bits * rows * row_words(k);
 }
 
-// ---- host-buffer fully-connected layer -----------------------------------------------------
+// ---- whole fully-connected layer (Fig. 1): device buffers, then host buffers -------------------
 namespace {
-struct LinearLayout {
-    int64_t x, w, s_a, s_w, a_planes, w_planes, out_i32, out_f32, total;
-};
 inline int64_t up256(int64_t v) { return (v + 255) / 256 * 256; }
-LinearLayout linear_layout(int64_t m, int64_t n, int64_t k, int a_bits, int w_bits) {
-    LinearLayout L;
+
+// Scratch of one layer call: both ranges and both packed operands.
+struct LinearScratch {
+    int64_t s_a, s_w, a_planes, w_planes, total;
+};
+LinearScratch linear_scratch(int64_t m, int64_t n, int64_t k, int a_bits, int w_bits) {
+    LinearScratch L;
     int64_t off = 0;
-    L.x = off; off += up256(m * k * 4);
-    L.w = off; off += up256(n * k * 4);
     L.s_a = off; off += 256;
     L.s_w = off; off += up256(n * 4);
     L.a_planes = off; off += up256(mpq_packed_words(m, k, a_bits) * 4);
     L.w_planes = off; off += up256(mpq_packed_words(n, k, w_bits) * 4);
-    L.out_i32 = off; off += up256(m * n * 4);
-    L.out_f32 = off; off += up256(m * n * 4);
     L.total = off;
     return L;
 }
+
+// Host staging of mpq_linear_host: fp32 operands and results, then the layer's own scratch.
+struct HostLayout {
+    int64_t x, w, out_i32, out_f32, scratch, total;
+};
+HostLayout host_layout(int64_t m, int64_t n, int64_t k, int a_bits, int w_bits) {
+    HostLayout L;
+    int64_t off = 0;
+    L.x = off; off += up256(m * k * 4);
+    L.w = off; off += up256(n * k * 4);
+    L.out_i32 = off; off += up256(m * n * 4);
+    L.out_f32 = off; off += up256(m * n * 4);
+    L.scratch = off; off += linear_scratch(m, n, k, a_bits, w_bits).total;
+    L.total = off;
+    return L;
+}
+
+int linear_args_ok(int64_t m, int64_t n, int64_t k, int a_bits, int w_bits, int a_act, int w_mode) {
+    if (m <= 0 || n <= 0 || k <= 0) return MPQ_ERR_BAD_SHAPE;
+    if (!bits_ok(a_bits) || !bits_ok(w_bits) || (a_act != MPQ_ACT_HTANH && a_act != MPQ_ACT_HRELU) ||
+        (w_mode != MPQ_SCALE_PER_TENSOR && w_mode != MPQ_SCALE_PER_ROW)) return MPQ_ERR_UNSUPPORTED;
+    return MPQ_OK;
+}
+
+// range -> encode -> product with the scratch at `ws` (256-byte aligned device memory)
+int linear_on_scratch(const float* x, const float* w, int64_t m, int64_t n, int64_t k,
+                      int a_bits, int w_bits, int a_act, int w_mode,
+                      int32_t* out_i32, float* out_f32, char* ws, cudaStream_t st) {
+    const LinearScratch L = linear_scratch(m, n, k, a_bits, w_bits);
+    float* s_a = reinterpret_cast<float*>(ws + L.s_a);
+    float* s_w = reinterpret_cast<float*>(ws + L.s_w);
+    uint32_t* ap = reinterpret_cast<uint32_t*>(ws + L.a_planes);
+    uint32_t* wp = reinterpret_cast<uint32_t*>(ws + L.w_planes);
+    int rc;
+    if ((rc = mpq_absmax(x, m, k, k, MPQ_SCALE_PER_TENSOR, a_act, s_a, st)) != MPQ_OK) return rc;
+    if ((rc = mpq_absmax(w, n, k, k, w_mode, MPQ_ACT_HTANH, s_w, st)) != MPQ_OK) return rc;
+    if ((rc = mpq_encode(x, m, k, k, s_a, MPQ_SCALE_PER_TENSOR, a_act, a_bits, ap, st)) != MPQ_OK) return rc;
+    if ((rc = mpq_encode(w, n, k, k, s_w, w_mode, MPQ_ACT_HTANH, w_bits, wp, st)) != MPQ_OK) return rc;
+    return mpq_gemm(ap, a_bits, wp, w_bits, m, n, k, out_i32, out_f32, n, s_a, s_w, w_mode, st);
+}
 }  // namespace
+
+extern "C" int64_t mpq_linear_workspace(int64_t m, int64_t n, int64_t k, int a_bits, int w_bits) {
+    if (m <= 0 || n <= 0 || k <= 0 || !bits_ok(a_bits) || !bits_ok(w_bits)) return 0;
+    return linear_scratch(m, n, k, a_bits, w_bits).total;
+}
+
+extern "C" int mpq_linear(const float* x, const float* w, int64_t m, int64_t n, int64_t k,
+                          int a_bits, int w_bits, int a_act, int w_mode,
+                          int32_t* out_i32, float* out_f32,
+                          void* workspace, int64_t workspace_bytes, void* stream) {
+    if (!x || !w || !workspace || (!out_i32 && !out_f32)) return MPQ_ERR_NULL;
+    const int rc = linear_args_ok(m, n, k, a_bits, w_bits, a_act, w_mode);
+    if (rc != MPQ_OK) return rc;
+    if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return MPQ_ERR_ALIGN;
+    if (workspace_bytes < linear_scratch(m, n, k, a_bits, w_bits).total) return MPQ_ERR_WORKSPACE;
+    return linear_on_scratch(x, w, m, n, k, a_bits, w_bits, a_act, w_mode, out_i32, out_f32,
+                             static_cast<char*>(workspace), (cudaStream_t)stream);
+}
 
 extern "C" int64_t mpq_linear_host_workspace(int64_t m, int64_t n, int64_t k, int a_bits, int w_bits) {
     if (m <= 0 || n <= 0 || k <= 0 || !bits_ok(a_bits) || !bits_ok(w_bits)) return 0;
-    return linear_layout(m, n, k, a_bits, w_bits).total;
+    return host_layout(m, n, k, a_bits, w_bits).total;
 }
 
 extern "C" int mpq_linear_host(const float* x_host, const float* w_host, int64_t m, int64_t n, int64_t k,
@@ -56,33 +112,22 @@ extern "C" int mpq_linear_host(const float* x_host, const float* w_host, int64_t
                                int32_t* out_i32_host, float* out_f32_host,
                                void* workspace, int64_t workspace_bytes, void* stream) {
     if (!x_host || !w_host || !workspace || (!out_i32_host && !out_f32_host)) return MPQ_ERR_NULL;
-    if (m <= 0 || n <= 0 || k <= 0) return MPQ_ERR_BAD_SHAPE;
-    if (!bits_ok(a_bits) || !bits_ok(w_bits)) return MPQ_ERR_UNSUPPORTED;
+    int rc = linear_args_ok(m, n, k, a_bits, w_bits, a_act, w_mode);
+    if (rc != MPQ_OK) return rc;
     if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return MPQ_ERR_ALIGN;
-    const LinearLayout L = linear_layout(m, n, k, a_bits, w_bits);
+    const HostLayout L = host_layout(m, n, k, a_bits, w_bits);
     if (workspace_bytes < L.total) return MPQ_ERR_WORKSPACE;
     cudaStream_t st = (cudaStream_t)stream;
     char* ws = static_cast<char*>(workspace);
     float* x = reinterpret_cast<float*>(ws + L.x);
     float* w = reinterpret_cast<float*>(ws + L.w);
-    float* s_a = reinterpret_cast<float*>(ws + L.s_a);
-    float* s_w = reinterpret_cast<float*>(ws + L.s_w);
-    uint32_t* ap = reinterpret_cast<uint32_t*>(ws + L.a_planes);
-    uint32_t* wp = reinterpret_cast<uint32_t*>(ws + L.w_planes);
-    int32_t* oi = reinterpret_cast<int32_t*>(ws + L.out_i32);
-    float* of = reinterpret_cast<float*>(ws + L.out_f32);
-
+    int32_t* oi = out_i32_host ? reinterpret_cast<int32_t*>(ws + L.out_i32) : nullptr;
+    float* of = out_f32_host ? reinterpret_cast<float*>(ws + L.out_f32) : nullptr;
     if (cudaMemcpyAsync(x, x_host, (size_t)m * k * 4, cudaMemcpyHostToDevice, st) != cudaSuccess) return MPQ_ERR_CUDA;
     if (cudaMemcpyAsync(w, w_host, (size_t)n * k * 4, cudaMemcpyHostToDevice, st) != cudaSuccess) return MPQ_ERR_CUDA;
-    int rc;
-    if ((rc = mpq_absmax(x, m, k, k, MPQ_SCALE_PER_TENSOR, a_act, s_a, st)) != MPQ_OK) return rc;
-    if ((rc = mpq_absmax(w, n, k, k, w_mode, MPQ_ACT_HTANH, s_w, st)) != MPQ_OK) return rc;
-    if ((rc = mpq_encode(x, m, k, k, s_a, MPQ_SCALE_PER_TENSOR, a_act, a_bits, ap, st)) != MPQ_OK) return rc;
-    if ((rc = mpq_encode(w, n, k, k, s_w, w_mode, MPQ_ACT_HTANH, w_bits, wp, st)) != MPQ_OK) return rc;
-    if ((rc = mpq_gemm(ap, a_bits, wp, w_bits, m, n, k, out_i32_host ? oi : nullptr, out_f32_host ? of : nullptr, n,
-                       s_a, s_w, w_mode, st)) != MPQ_OK) return rc;
-    if (out_i32_host && cudaMemcpyAsync(out_i32_host, oi, (size_t)m * n * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess) return MPQ_ERR_CUDA;
-    if (out_f32_host && cudaMemcpyAsync(out_f32_host, of, (size_t)m * n * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess) return MPQ_ERR_CUDA;
+    if ((rc = linear_on_scratch(x, w, m, n, k, a_bits, w_bits, a_act, w_mode, oi, of, ws + L.scratch, st)) != MPQ_OK) return rc;
+    if (oi && cudaMemcpyAsync(out_i32_host, oi, (size_t)m * n * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess) return MPQ_ERR_CUDA;
+    if (of && cudaMemcpyAsync(out_f32_host, of, (size_t)m * n * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess) return MPQ_ERR_CUDA;
     return cudaStreamSynchronize(st) == cudaSuccess ? MPQ_OK : MPQ_ERR_CUDA;
 }
 

@@ -84,7 +84,13 @@ def test_host_side_argument_checks(mpq):
     assert conv(a_bits=8, w_bits=8, C=4096) == ERR_OVER    # 9 * 4096 * 255 * 255 >= 2^31
     assert L.mpq_encode_nchw(aligned, 1, 48, 4, 4, aligned, 0, 2, aligned, NULL) == ERR_UNSUP
     assert L.mpq_encode_oihw(aligned, 4, 64, 3, 3, aligned, 0, 2, aligned, NULL, NULL) == ERR_NULL
-    # host-buffer layer
+    # whole-layer calls
+    assert mpq.linear_workspace(4, 0, 4, 2, 2) == 0
+    lw = mpq.linear_workspace(64, 64, 512, 2, 2)
+    assert lw >= 2 * 2 * 64 * 16 * 4
+    assert L.mpq_linear(aligned, aligned, 64, 64, 512, 2, 2, 0, 0, aligned, NULL, ctypes.c_void_p(256), lw - 1, NULL) == 7
+    assert L.mpq_linear(aligned, aligned, 64, 64, 512, 2, 2, 0, 0, aligned, NULL, ctypes.c_void_p(260), lw, NULL) == ERR_ALIGN
+    assert L.mpq_linear(aligned, aligned, 64, 64, 512, 2, 9, 0, 0, aligned, NULL, ctypes.c_void_p(256), lw, NULL) == ERR_UNSUP
     assert mpq.linear_host_workspace(0, 4, 4, 2, 2) == 0
     need = mpq.linear_host_workspace(64, 64, 512, 2, 2)
     assert need >= 2 * 64 * 512 * 4 + 2 * 64 * 64 * 4

@@ -287,7 +287,20 @@ def test_conv_1x1_equals_gemm(mpq, cuda):
     assert np.array_equal(yi.cpu().numpy().transpose(0, 2, 3, 1).reshape(60, 24), ci.cpu().numpy())
 
 
-# ---------------------------------------------------------------------------- host-buffer layer
+# ---------------------------------------------------------------------------- whole-layer calls
+@pytest.mark.parametrize("m,n,k,a_bits,w_bits,per_row", [(64, 64, 512, 2, 2, False), (33, 70, 1000, 3, 4, True)])
+def test_linear_device(mpq, cuda, m, n, k, a_bits, w_bits, per_row):
+    rng = np.random.default_rng(m + n)
+    x = np.maximum(rng.standard_normal((m, k)), 0).astype(np.float32)
+    w = rng.standard_normal((n, k)).astype(np.float32)
+    oi = torch.empty((m, n), dtype=torch.int32, device=cuda)
+    of = torch.empty((m, n), dtype=torch.float32, device=cuda)
+    mpq.linear(_dev(x, cuda), _dev(w, cuda), a_bits, w_bits, mpq.ACT_HRELU, int(per_row), oi, of)
+    acc_ref, out_ref, _, _ = oracle.linear(x, w, a_bits, w_bits, w_per_row=per_row, a_act=oracle.HRELU)
+    assert np.array_equal(oi.cpu().numpy(), acc_ref)
+    assert rel_close(of.cpu().numpy(), out_ref)
+
+
 def test_linear_host(mpq, cuda):
     c = inputs.config1()
     x = torch.from_numpy(c["x"]).pin_memory()
