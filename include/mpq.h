@@ -46,7 +46,8 @@ typedef enum {
     MPQ_ERR_OVERFLOW = 4,    /* k * (2^a_bits-1) * (2^w_bits-1) >= 2^31: int32 would overflow */
     MPQ_ERR_ALIGN = 5,       /* a plane pointer is not 16-byte aligned                       */
     MPQ_ERR_CUDA = 6,        /* the CUDA runtime reported an error (launch, copy)            */
-    MPQ_ERR_WORKSPACE = 7    /* caller-provided workspace is too small                       */
+    MPQ_ERR_WORKSPACE = 7,   /* caller-provided workspace is too small                       */
+    MPQ_ERR_STATIC_LIMIT = 8 /* problem needs more than the library's built-in scratch       */
 } mpq_status;
 
 typedef enum { MPQ_SCALE_PER_TENSOR = 0, MPQ_SCALE_PER_ROW = 1 } mpq_scale_mode;
@@ -134,6 +135,30 @@ int mpq_linear(const float* x, const float* w, int64_t m, int64_t n, int64_t k,
                int a_bits, int w_bits, int a_act, int w_mode,
                int32_t* out_i32, float* out_f32,
                void* workspace, int64_t workspace_bytes, void* stream);
+
+/* ---- The same layer for callers that cannot allocate device memory.  (The paper has no
+ * counterpart: this is a packaging variant of mpq_linear, same arithmetic, same results.)
+ * Some users of this library may not call cudaMalloc at the point where they need a layer:
+ * an inference plug-in running inside a host framework that has already claimed the device's
+ * memory for its own pool, a service whose start-up phase is the only place allocation is
+ * allowed (cudaMalloc can block on the whole device and can fail late), or a small embedding
+ * program that has no allocator to lend a workspace from.  For them the two ranges and the two
+ * packed operands live in a buffer that is part of the library image itself: a file-scope
+ * device array of MPQ_LINEAR_STATIC_BYTES bytes that every GPU which loads libmpq.so holds
+ * until the process exits.  The caller passes only inputs and outputs (device pointers, as for
+ * mpq_linear).  Nothing is allocated or freed, here or in anything this call uses.
+ *   - Limit: mpq_linear_workspace(m, n, k, a_bits, w_bits) must not exceed
+ *     MPQ_LINEAR_STATIC_BYTES, else MPQ_ERR_STATIC_LIMIT is returned and nothing is launched.
+ *   - The first call on each device looks up the buffer's device address (with that device
+ *     current) and remembers it; make that first call outside any stream capture.
+ *   - All calls on a device share the one buffer, and it keeps whatever the previous call left.
+ *     Nothing in it has to start at zero except the range words, which the range step clears on
+ *     the stream itself.  Two calls that overlap on the GPU (different streams, or different
+ *     host threads without ordering between their streams) race on the buffer: serialise them. */
+#define MPQ_LINEAR_STATIC_BYTES (16 * 1024 * 1024)
+int mpq_linear_static(const float* x, const float* w, int64_t m, int64_t n, int64_t k,
+                      int a_bits, int w_bits, int a_act, int w_mode,
+                      int32_t* out_i32, float* out_f32, void* stream);
 
 /* The same layer from HOST buffers: copies x_host and w_host into the device workspace, runs
  * mpq_linear there, and copies out_i32_host / out_f32_host [m x n] back (either may be NULL, not

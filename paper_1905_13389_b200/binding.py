@@ -55,13 +55,14 @@ def lib() -> ctypes.CDLL:
         L.mpq_linear_workspace.argtypes = [i64, i64, i64, i32, i32]
         L.mpq_linear_workspace.restype = i64
         L.mpq_linear.argtypes = [P, P, i64, i64, i64, i32, i32, i32, i32, P, P, P, i64, P]
+        L.mpq_linear_static.argtypes = [P, P, i64, i64, i64, i32, i32, i32, i32, P, P, P]
         L.mpq_linear_host_workspace.argtypes = [i64, i64, i64, i32, i32]
         L.mpq_linear_host_workspace.restype = i64
         L.mpq_linear_host.argtypes = [P, P, i64, i64, i64, i32, i32, i32, i32, P, P, P, i64, P]
         L.mpq_measure_popc_peak.argtypes = [ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double),
                                             ctypes.POINTER(ctypes.c_int), P]
         for name in ("mpq_absmax", "mpq_encode", "mpq_encode_nchw", "mpq_encode_oihw", "mpq_gemm", "mpq_conv",
-                     "mpq_add_relu", "mpq_linear", "mpq_linear_host", "mpq_measure_popc_peak"):
+                     "mpq_add_relu", "mpq_linear", "mpq_linear_static", "mpq_linear_host", "mpq_measure_popc_peak"):
             getattr(L, name).restype = i32
         _lib = L
     return _lib
@@ -195,6 +196,23 @@ def linear(x: torch.Tensor, w: torch.Tensor, a_bits: int, w_bits: int,
     _check(lib().mpq_linear(_ptr(x, torch.float32), _ptr(w, torch.float32), m, n, k, a_bits, w_bits, a_act, w_mode,
                             _ptr(out_i32, torch.int32), _ptr(out_f32, torch.float32),
                             workspace.data_ptr(), workspace.numel(), _stream()), "mpq_linear")
+    return out_i32, out_f32
+
+
+LINEAR_STATIC_BYTES = 16 * 1024 * 1024
+
+
+def linear_static(x: torch.Tensor, w: torch.Tensor, a_bits: int, w_bits: int,
+                  a_act: int = ACT_HTANH, w_mode: int = SCALE_PER_TENSOR,
+                  out_i32: Optional[torch.Tensor] = None, out_f32: Optional[torch.Tensor] = None):
+    """:func:`linear` for callers that may not allocate: the ranges and packed operands go to a
+    buffer built into the library (LINEAR_STATIC_BYTES per GPU) instead of a workspace tensor.
+    Calls on one device share that buffer, so do not let two of them overlap on the GPU."""
+    m, k = x.shape
+    n, _ = w.shape
+    _check(lib().mpq_linear_static(_ptr(x, torch.float32), _ptr(w, torch.float32), m, n, k, a_bits, w_bits,
+                                   a_act, w_mode, _ptr(out_i32, torch.int32), _ptr(out_f32, torch.float32),
+                                   _stream()), "mpq_linear_static")
     return out_i32, out_f32
 
 

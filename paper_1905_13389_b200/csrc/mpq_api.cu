@@ -1,4 +1,6 @@
 // Status strings, size queries, the host-buffer fully-connected layer and the POPC-rate probe.
+#include <mutex>
+
 #include "mpq_common.cuh"
 
 using namespace mpq;
@@ -13,6 +15,7 @@ extern "C" const char* mpq_status_string(int status) {
         case MPQ_ERR_ALIGN: return "pointer not 16-byte aligned";
         case MPQ_ERR_CUDA: return "CUDA runtime error";
         case MPQ_ERR_WORKSPACE: return "workspace too small";
+        case MPQ_ERR_STATIC_LIMIT: return "problem needs more scratch than MPQ_LINEAR_STATIC_BYTES";
     }
     return "unknown status";
 }
@@ -100,6 +103,46 @@ extern "C" int mpq_linear(const float* x, const float* w, int64_t m, int64_t n, 
     if (workspace_bytes < linear_scratch(m, n, k, a_bits, w_bits).total) return MPQ_ERR_WORKSPACE;
     return linear_on_scratch(x, w, m, n, k, a_bits, w_bits, a_act, w_mode, out_i32, out_f32,
                              static_cast<char*>(workspace), (cudaStream_t)stream);
+}
+
+// ---- the layer on the library's own scratch: no allocation anywhere --------------------------
+// The scratch is part of the loaded module: each GPU that loads the library carries these
+// MPQ_LINEAR_STATIC_BYTES until the process exits.  In host code the array's name is only a
+// handle for cudaGetSymbolAddress; kernels must be given the address that call returns.
+static __device__ __align__(256) unsigned char g_linear_static_scratch[MPQ_LINEAR_STATIC_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mutex;
+unsigned char* g_static_ptr[kMaxDevices] = {};   // device address of the scratch, per device
+
+// Looked up once per device, with that device current (the caller's current device).
+int static_scratch_address(unsigned char** out) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return MPQ_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    if (!g_static_ptr[dev]) {
+        void* ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_linear_static_scratch) != cudaSuccess || !ptr) return MPQ_ERR_CUDA;
+        g_static_ptr[dev] = static_cast<unsigned char*>(ptr);
+    }
+    *out = g_static_ptr[dev];
+    return MPQ_OK;
+}
+}  // namespace
+
+extern "C" int mpq_linear_static(const float* x, const float* w, int64_t m, int64_t n, int64_t k,
+                                 int a_bits, int w_bits, int a_act, int w_mode,
+                                 int32_t* out_i32, float* out_f32, void* stream) {
+    if (!x || !w || (!out_i32 && !out_f32)) return MPQ_ERR_NULL;
+    int rc = linear_args_ok(m, n, k, a_bits, w_bits, a_act, w_mode);
+    if (rc != MPQ_OK) return rc;
+    if (linear_scratch(m, n, k, a_bits, w_bits).total > (int64_t)MPQ_LINEAR_STATIC_BYTES) return MPQ_ERR_STATIC_LIMIT;
+    unsigned char* scratch = nullptr;
+    if ((rc = static_scratch_address(&scratch)) != MPQ_OK) return rc;
+    // Ranges are cleared by the range step on the stream; planes are fully rewritten by the encoders.
+    return linear_on_scratch(x, w, m, n, k, a_bits, w_bits, a_act, w_mode, out_i32, out_f32,
+                             reinterpret_cast<char*>(scratch), (cudaStream_t)stream);
 }
 
 extern "C" int64_t mpq_linear_host_workspace(int64_t m, int64_t n, int64_t k, int a_bits, int w_bits) {
