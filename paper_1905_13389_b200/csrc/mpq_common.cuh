@@ -34,4 +34,56 @@ __device__ __forceinline__ int level_index(float x, float inv_s, float half_L, f
     return __float2int_rd(y) + H;
 }
 
+// ---- The quantizer and the bit-plane split on the floating-point pipe ---------------------
+// level_fraction() returns z in [0, 1) with  u = floor(2^BITS * z)  (HReLU: u = H + floor(2^BITS * z)),
+// H = 2^(BITS-1), u the level index of level_index():
+//   HTanh: z = min(sat(RD(y/2H + 1/2)), 1 - 1/4H)        HReLU: z = min(sat(y/2H), 1/2 - 1/4H)
+// sat() clamps to [0,1] inside the multiply-add; the round-down addition keeps a value that lies
+// just below a level boundary below it (n/2H is representable, so floor(2H*RD(t)) = floor(2H*t)).
+// Equal to level_index() for every input except a NaN under HTanh (sat() sends a NaN to 0, not
+// to the level above zero): callers look for NaNs themselves and fall back to level_index().
+template <int BITS, int ACT>
+__device__ __forceinline__ float level_fraction(float x, float inv_s, float half_L) {
+    constexpr float kInvTwoH = 1.0f / (float)(1 << BITS);
+    const float y = __fmul_rn(__fmul_rn(x, inv_s), half_L);
+    float z;
+    if (ACT == MPQ_ACT_HRELU) {
+        asm("mul.rn.sat.f32 %0, %1, %2;" : "=f"(z) : "f"(y), "f"(kInvTwoH));
+        return fminf(z, 0.5f - 0.5f * kInvTwoH);
+    }
+    asm("fma.rm.sat.f32 %0, %1, %2, %3;" : "=f"(z) : "f"(y), "f"(kInvTwoH), "f"(0.5f));
+    return fminf(z, 1.0f - 0.5f * kInvTwoH);
+}
+
+// Builds, in one thread, the BITS plane words of 32 elements pushed from element 31 down to
+// element 0, without a per-bit test: for plane p the value floor(u / 2^p) drops out of one
+// round-down multiply-add (2^23 is added so that the integer sits in the low mantissa bits),
+//     t_p = bits(RD(z * 2^(BITS-p) + 2^23 + (H >> p)))  =  0x4B000000 + floor(u / 2^p),
+// it is shifted in with  acc_p = 2 acc_p + t_p  (arithmetic mod 2^32, so the running sums may
+// wrap), and since bit p of u is floor(u/2^p) - 2 floor(u/2^(p+1)) the plane words are
+//     word_p = T_p - 2 T_(p+1),   T_p = acc_p + 0x4B000000,   T_BITS = 0
+// (the 32 added constants sum to 0x4B000000 * (2^32 - 1) = -0x4B000000).  `two` is the number 2
+// passed in a register: a multiplier the compiler cannot see keeps the doubling an integer
+// multiply-add on the FMA pipe instead of a shift-add on the (busier) integer ALU.
+template <int BITS, int ACT>
+struct LaneWords {
+    uint32_t acc[BITS];
+    __device__ __forceinline__ void clear() {
+#pragma unroll
+        for (int p = 0; p < BITS; ++p) acc[p] = 0u;
+    }
+    __device__ __forceinline__ void push(float z, uint32_t two) {
+#pragma unroll
+        for (int p = 0; p < BITS; ++p) {
+            const float magic = 8388608.0f + (ACT == MPQ_ACT_HRELU ? (float)((1 << (BITS - 1)) >> p) : 0.0f);
+            const uint32_t t = __float_as_uint(__fmaf_rd(z, (float)(1 << (BITS - p)), magic));
+            acc[p] = acc[p] * two + t;
+        }
+    }
+    __device__ __forceinline__ uint32_t word(int p) const {
+        const uint32_t T = acc[p] + 0x4B000000u;
+        return p + 1 < BITS ? T - 2u * (acc[p + 1] + 0x4B000000u) : T;
+    }
+};
+
 }  // namespace mpq

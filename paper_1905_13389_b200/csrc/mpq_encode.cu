@@ -59,18 +59,38 @@ absmax_kernel(const float* __restrict__ x, int64_t k, int64_t ldx, int64_t chunk
 }
 
 // ------------------------------------------------------------------------------------------
-// Row-major encoder.  One warp packs 1024 consecutive elements of a row (32 words per plane):
-// in step j lane L quantizes element 32 j + L (a fully coalesced 128-byte read), one
-// __ballot_sync per plane transposes that bit across the warp into word j, and lane j keeps it,
-// so the final store of each plane is again one coalesced 128-byte write.
+// Row-major encoder.  One warp packs 1024 consecutive elements of a row (32 words per plane).
+//
+// Full, 16-byte aligned segments take the lane-local path: the 4 KiB segment is copied into
+// shared memory with coalesced 16-byte asynchronous copies (rows of 32 floats, padded to 36 so
+// that the later 16-byte reads of a quarter-warp fall in distinct banks), then lane L owns
+// elements 32 L .. 32 L + 31, i.e. word L of every plane, and builds its words with LaneWords:
+// the quantizer and the bit split run on the floating-point pipe, the integer ALU sees one min
+// per element, and the plane stores are coalesced 128-byte rows.  The kernel is then limited by
+// HBM, not by issue slots.  A lane that meets a NaN (HTanh) or a degenerate range rebuilds its
+// words with the plain quantizer.
+//
+// Ragged or unaligned segments take the ballot path: in step j lane L quantizes element
+// 32 j + L and one __ballot_sync per plane transposes that bit across the warp into word j.
 // ------------------------------------------------------------------------------------------
 constexpr int kEncodeThreads = 256;
+constexpr int kStageRow = 36;          // floats per staged 32-float row (16 bytes of padding)
+
+__device__ __forceinline__ void copy_async_16(void* smem_dst, const void* gsrc) {
+    const unsigned dst = (unsigned)__cvta_generic_to_shared(smem_dst);
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(dst), "l"(gsrc) : "memory");
+}
+__device__ __forceinline__ void copy_async_wait_all() {
+    asm volatile("cp.async.commit_group;\ncp.async.wait_group 0;\n" ::: "memory");
+}
 
 template <int BITS, int ACT>
 __global__ void __launch_bounds__(kEncodeThreads)
 encode_rows_kernel(const float* __restrict__ x, int64_t rows, int64_t k, int64_t ldx,
                    const float* __restrict__ scale, int per_row,
-                   uint32_t* __restrict__ planes, int64_t rw, int64_t segs_per_row) {
+                   uint32_t* __restrict__ planes, int64_t rw, int64_t segs_per_row,
+                   int vec_ok, uint32_t two) {
+    __shared__ __align__(16) float stage[kEncodeThreads / 32][32 * kStageRow];
     const int64_t warp = (int64_t)blockIdx.x * (kEncodeThreads / 32) + (threadIdx.x >> 5);
     if (warp >= rows * segs_per_row) return;
     const int lane = threadIdx.x & 31;
@@ -83,12 +103,53 @@ encode_rows_kernel(const float* __restrict__ x, int64_t rows, int64_t k, int64_t
     const float half_L = 0.5f * (float)((1 << BITS) - 1);
     const float lo = (float)(-H), hi = (float)H - 0.5f;
     const float inv = inverse_scale(__ldg(scale + (per_row ? row : 0)));
+    const int64_t remaining = k - e0;                       // > 0 only for words that hold data
+
+    if (vec_ok && remaining >= 1024) {
+        float* mine = stage[threadIdx.x >> 5];
+        const float* src = xr + e0;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const int chunk = 32 * i + lane;                // 16-byte chunk of the segment
+            copy_async_16(mine + (chunk >> 3) * kStageRow + (chunk & 7) * 4, src + chunk * 4);
+        }
+        copy_async_wait_all();
+        __syncwarp();
+        const float4* own = reinterpret_cast<const float4*>(mine + lane * kStageRow);
+        LaneWords<BITS, ACT> lw;
+        lw.clear();
+        float probe = 0.0f;                                 // turns NaN if any element is NaN
+#pragma unroll
+        for (int c = 7; c >= 0; --c) {
+            const float4 v = own[c];
+            if (ACT == MPQ_ACT_HTANH) probe = fmaf(v.x, v.y, fmaf(v.z, v.w, probe));
+            lw.push(level_fraction<BITS, ACT>(v.w, inv, half_L), two);
+            lw.push(level_fraction<BITS, ACT>(v.z, inv, half_L), two);
+            lw.push(level_fraction<BITS, ACT>(v.y, inv, half_L), two);
+            lw.push(level_fraction<BITS, ACT>(v.x, inv, half_L), two);
+        }
+        uint32_t word[BITS];
+#pragma unroll
+        for (int p = 0; p < BITS; ++p) word[p] = lw.word(p);
+        if (ACT == MPQ_ACT_HTANH && (probe != probe || inv == 0.0f)) {
+#pragma unroll
+            for (int p = 0; p < BITS; ++p) word[p] = 0u;
+            for (int t = 0; t < 32; ++t) {
+                const uint32_t u = (uint32_t)level_index<ACT>(mine[lane * kStageRow + t], inv, half_L, lo, hi, H);
+#pragma unroll
+                for (int p = 0; p < BITS; ++p) word[p] |= ((u >> p) & 1u) << t;
+            }
+        }
+        uint32_t* dst = planes + row * rw + seg * 32 + lane;
+        const int64_t plane_stride = rows * rw;
+#pragma unroll
+        for (int p = 0; p < BITS; ++p) dst[p * plane_stride] = word[p];
+        return;
+    }
 
     uint32_t mine[BITS];
 #pragma unroll
     for (int p = 0; p < BITS; ++p) mine[p] = 0u;
-
-    const int64_t remaining = k - e0;                       // > 0 only for words that hold data
     const int steps = remaining >= 1024 ? 32 : (int)((remaining + 31) / 32);   // warp-uniform
     for (int j0 = 0; j0 < steps; j0 += 8) {
         float v[8];
@@ -119,13 +180,13 @@ encode_rows_kernel(const float* __restrict__ x, int64_t rows, int64_t k, int64_t
 // ------------------------------------------------------------------------------------------
 // NCHW activations -> planes[bits][N][H][W][C/32].  A warp takes 32 pixels x 32 channels:
 // lane = pixel, so each of the 32 channel reads is a coalesced 128-byte row of one channel,
-// and every lane builds the word of its own pixel bit by bit (channel c -> bit c).
+// and every lane builds the word of its own pixel (channel c -> bit c) with LaneWords.
 // ------------------------------------------------------------------------------------------
 template <int BITS, int ACT>
 __global__ void __launch_bounds__(kEncodeThreads)
 encode_nchw_kernel(const float* __restrict__ x, int N, int C, int64_t HW,
                    const float* __restrict__ scale, uint32_t* __restrict__ planes,
-                   int64_t pix_blocks, int64_t total_warps) {
+                   int64_t pix_blocks, int64_t total_warps, uint32_t two) {
     const int64_t warp = (int64_t)blockIdx.x * (kEncodeThreads / 32) + (threadIdx.x >> 5);
     if (warp >= total_warps) return;
     const int lane = threadIdx.x & 31;
@@ -135,7 +196,7 @@ encode_nchw_kernel(const float* __restrict__ x, int N, int C, int64_t HW,
     const int cw = (int)(rest % Cw);
     const int64_t n = rest / Cw;
     const int64_t pixel = pb * 32 + lane;
-    const bool valid = pixel < HW;
+    if (pixel >= HW) return;
 
     constexpr int H = 1 << (BITS - 1);
     const float half_L = 0.5f * (float)((1 << BITS) - 1);
@@ -143,26 +204,35 @@ encode_nchw_kernel(const float* __restrict__ x, int N, int C, int64_t HW,
     const float inv = inverse_scale(__ldg(scale));
 
     const float* base = x + ((n * C + (int64_t)cw * 32) * HW + pixel);
-    uint32_t word[BITS];
+    LaneWords<BITS, ACT> lw;
+    lw.clear();
+    float probe = 0.0f;                                     // turns NaN if any element is NaN
 #pragma unroll
-    for (int p = 0; p < BITS; ++p) word[p] = 0u;
-#pragma unroll
-    for (int c0 = 0; c0 < 32; c0 += 8) {
+    for (int c0 = 24; c0 >= 0; c0 -= 8) {
         float v[8];
 #pragma unroll
-        for (int cc = 0; cc < 8; ++cc) v[cc] = valid ? __ldg(base + (int64_t)(c0 + cc) * HW) : 0.0f;
+        for (int cc = 0; cc < 8; ++cc) v[cc] = __ldg(base + (int64_t)(c0 + cc) * HW);
 #pragma unroll
-        for (int cc = 0; cc < 8; ++cc) {
-            const uint32_t u = (uint32_t)level_index<ACT>(v[cc], inv, half_L, lo, hi, H);
-#pragma unroll
-            for (int p = 0; p < BITS; ++p) word[p] |= ((u >> p) & 1u) << (c0 + cc);
+        for (int cc = 7; cc >= 0; --cc) {
+            if (ACT == MPQ_ACT_HTANH && (cc & 1)) probe = fmaf(v[cc], v[cc - 1], probe);
+            lw.push(level_fraction<BITS, ACT>(v[cc], inv, half_L), two);
         }
     }
-    if (valid) {
+    uint32_t word[BITS];
 #pragma unroll
-        for (int p = 0; p < BITS; ++p)
-            planes[(((int64_t)p * N + n) * HW + pixel) * Cw + cw] = word[p];
+    for (int p = 0; p < BITS; ++p) word[p] = lw.word(p);
+    if (ACT == MPQ_ACT_HTANH && (probe != probe || inv == 0.0f)) {
+#pragma unroll
+        for (int p = 0; p < BITS; ++p) word[p] = 0u;
+        for (int c = 0; c < 32; ++c) {
+            const uint32_t u = (uint32_t)level_index<ACT>(__ldg(base + (int64_t)c * HW), inv, half_L, lo, hi, H);
+#pragma unroll
+            for (int p = 0; p < BITS; ++p) word[p] |= ((u >> p) & 1u) << c;
+        }
     }
+#pragma unroll
+    for (int p = 0; p < BITS; ++p)
+        planes[(((int64_t)p * N + n) * HW + pixel) * Cw + cw] = word[p];
 }
 
 // ------------------------------------------------------------------------------------------
@@ -241,8 +311,10 @@ struct EncodeRowsLauncher {
         const int64_t warps = rows * segs;
         const int64_t blocks = ceil_div(warps, kEncodeThreads / 32);
         if (blocks > 0x7fffffffLL) return MPQ_ERR_BAD_SHAPE;
+        // the lane-local path copies 16-byte chunks: every row start must be 16-byte aligned
+        const int vec_ok = aligned16(x) && (ldx % 4 == 0 || rows == 1);
         encode_rows_kernel<BITS, ACT><<<(unsigned)blocks, kEncodeThreads, 0, st>>>(
-            x, rows, k, ldx, scale, per_row, planes, rw, segs);
+            x, rows, k, ldx, scale, per_row, planes, rw, segs, vec_ok, 2u);
         return launch_status();
     }
 };
@@ -255,7 +327,7 @@ struct EncodeNchwLauncher {
         const int64_t blocks = ceil_div(warps, kEncodeThreads / 32);
         if (blocks > 0x7fffffffLL) return MPQ_ERR_BAD_SHAPE;
         encode_nchw_kernel<BITS, ACT><<<(unsigned)blocks, kEncodeThreads, 0, st>>>(
-            x, N, C, HW, scale, planes, pix_blocks, warps);
+            x, N, C, HW, scale, planes, pix_blocks, warps, 2u);
         return launch_status();
     }
 };

@@ -91,14 +91,38 @@ def test_encode_degenerate_scale(mpq, cuda):
         assert u.tolist() == [[4] * 6]                    # q = +1 everywhere
 
 
+@pytest.mark.parametrize("bits", [1, 2, 4, 7])
+def test_encode_rows_full_segments_with_specials(mpq, cuda, bits):
+    """Full 1024-element segments (the lean path) holding NaN, +-inf, exact ties, values far
+    outside the range and values one ulp either side of every level boundary."""
+    rng = np.random.default_rng(bits)
+    rows, k = 6, 3 * 1024 + 100
+    x = (rng.standard_normal((rows, k)) * 0.6).astype(np.float32)
+    L = 2 ** bits - 1
+    edges = np.array([(2 * n - L - 1) / L for n in range(0, L + 2)], dtype=np.float32)   # level boundaries
+    near = np.concatenate([edges, np.nextafter(edges, np.float32(9)), np.nextafter(edges, np.float32(-9))])
+    x[0, : near.size] = near
+    x[1, 5] = np.nan; x[1, 1500] = np.nan; x[2, 2047] = np.inf; x[2, 2048] = -np.inf
+    x[3, ::3] = 0.0; x[4, 10] = 1e30; x[4, 11] = -1e30; x[5, 7] = np.float32(1e-42); x[5, 8] = np.float32(-1e-42)
+    xd = _dev(x, cuda)
+    for act in (mpq.ACT_HTANH, mpq.ACT_HRELU):
+        for s in (np.ones(1, np.float32), np.array([0.37], np.float32), np.array([np.nan], np.float32)):
+            planes = mpq.encode(xd, _dev(s, cuda), bits, 0, act)
+            u = unpack_planes(planes.cpu().numpy(), k)
+            assert np.array_equal(u, oracle.levels(oracle.quantize(x, s, bits, act=act), bits))
+
+
 @pytest.mark.parametrize("bits", [1, 2, 3, 4, 8])
 @pytest.mark.parametrize("shape", [(2, 32, 5, 7), (1, 64, 9, 9), (3, 128, 4, 6), (2, 256, 14, 14)])
 def test_encode_nchw_codes(mpq, cuda, bits, shape):
     rng = np.random.default_rng(bits + shape[1])
     x = rng.standard_normal(shape).astype(np.float32)
     N, C, H, W = shape
+    x[0, 3, 1, 2] = np.nan; x[0, 5, 0, 0] = np.inf; x[0, 6, 0, 0] = -np.inf; x[:, 7] = 0.0
     for act in (mpq.ACT_HTANH, mpq.ACT_HRELU):
         s = oracle.absmax(x, False, act)
+        if not np.isfinite(s[0]):
+            s = np.ones(1, np.float32)
         planes = mpq.encode_nchw(_dev(x, cuda), _dev(s, cuda), bits, act).cpu().numpy()
         u = unpack_planes(planes.reshape(bits, N * H * W, C // 32), C).reshape(N, H, W, C).transpose(0, 3, 1, 2)
         assert np.array_equal(u, oracle.levels(oracle.quantize(x, s, bits, act=act), bits))
