@@ -123,6 +123,15 @@ int mpq_conv(const uint32_t* x_planes, int a_bits, int N, int C, int H, int W,
  * b may be NULL (plain ReLU).  n elements, fp32, one rounded add. */
 int mpq_add_relu(const float* a, const float* b, float* y, int64_t n, void* stream);
 
+/* ---- Full-precision glue of a ResNet-shaped stack (not part of the paper's method; the first
+ * layer of the network stays fp32).  Stem: x [N][3][H][W], w [64][3][7][7] -> y [N][64][Ho][Wo],
+ * 7x7, stride 2, zero pad 3, Ho = (H - 1)/2 + 1; relu != 0 applies max(.,0) in the store.  Each
+ * output is one chain of fused multiply-adds over (c, kh, kw) in that order.
+ * Max-pool: 3x3, stride 2, pad 1: x [N][C][H][W] -> y [N][C][(H - 1)/2 + 1][(W - 1)/2 + 1]. */
+int mpq_stem_conv7x7(const float* x, const float* w, float* y, int N, int H, int W, int relu,
+                     void* stream);
+int mpq_maxpool3x3s2(const float* x, float* y, int N, int C, int H, int W, void* stream);
+
 /* ---- Whole encoded fully-connected layer (Fig. 1 end to end: Encoder of both operands,
  * the a_bits x w_bits branches, Decoder): out = decode(encode(x) . encode(w)^T).
  * x [m x k] and w [n x k] are dense fp32 DEVICE tensors; activations take one range with `a_act`,

@@ -52,6 +52,8 @@ def lib() -> ctypes.CDLL:
         L.mpq_gemm.argtypes = [P, i32, P, i32, i64, i64, i64, P, P, i64, P, P, i32, P]
         L.mpq_conv.argtypes = [P, i32, i32, i32, i32, i32, P, i32, P, i32, i32, i32, i32, i32, P, P, P, P, i32, P]
         L.mpq_add_relu.argtypes = [P, P, P, i64, P]
+        L.mpq_stem_conv7x7.argtypes = [P, P, P, i32, i32, i32, i32, P]
+        L.mpq_maxpool3x3s2.argtypes = [P, P, i32, i32, i32, i32, P]
         L.mpq_linear_workspace.argtypes = [i64, i64, i64, i32, i32]
         L.mpq_linear_workspace.restype = i64
         L.mpq_linear.argtypes = [P, P, i64, i64, i64, i32, i32, i32, i32, P, P, P, i64, P]
@@ -62,7 +64,7 @@ def lib() -> ctypes.CDLL:
         L.mpq_measure_popc_peak.argtypes = [ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double),
                                             ctypes.POINTER(ctypes.c_int), P]
         for name in ("mpq_absmax", "mpq_encode", "mpq_encode_nchw", "mpq_encode_oihw", "mpq_gemm", "mpq_conv",
-                     "mpq_add_relu", "mpq_linear", "mpq_linear_static", "mpq_linear_host", "mpq_measure_popc_peak"):
+                     "mpq_add_relu", "mpq_stem_conv7x7", "mpq_maxpool3x3s2", "mpq_linear", "mpq_linear_static", "mpq_linear_host", "mpq_measure_popc_peak"):
             getattr(L, name).restype = i32
         _lib = L
     return _lib
@@ -178,6 +180,29 @@ def add_relu(a: torch.Tensor, b: Optional[torch.Tensor], y: torch.Tensor) -> tor
     _check(lib().mpq_add_relu(_ptr(a, torch.float32), _ptr(b, torch.float32), _ptr(y, torch.float32),
                               a.numel(), _stream()), "mpq_add_relu")
     return y
+
+
+def stem_conv7x7(x: torch.Tensor, w: torch.Tensor, relu: bool = True,
+                 out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """fp32 stem: x [N][3][H][W], w [64][3][7][7] -> [N][64][Ho][Wo] (7x7, stride 2, pad 3)."""
+    N, C, H, W = x.shape
+    if C != 3 or tuple(w.shape) != (64, 3, 7, 7):
+        raise ValueError("the stem takes 3 input channels and a [64][3][7][7] weight")
+    if out is None:
+        out = torch.empty((N, 64, (H - 1) // 2 + 1, (W - 1) // 2 + 1), dtype=torch.float32, device=x.device)
+    _check(lib().mpq_stem_conv7x7(_ptr(x, torch.float32), _ptr(w, torch.float32), _ptr(out, torch.float32),
+                                  N, H, W, int(relu), _stream()), "mpq_stem_conv7x7")
+    return out
+
+
+def maxpool3x3s2(x: torch.Tensor, out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """3x3 max-pool, stride 2, pad 1 on [N][C][H][W]."""
+    N, C, H, W = x.shape
+    if out is None:
+        out = torch.empty((N, C, (H - 1) // 2 + 1, (W - 1) // 2 + 1), dtype=torch.float32, device=x.device)
+    _check(lib().mpq_maxpool3x3s2(_ptr(x, torch.float32), _ptr(out, torch.float32), N, C, H, W, _stream()),
+           "mpq_maxpool3x3s2")
+    return out
 
 
 def linear_workspace(m: int, n: int, k: int, a_bits: int, w_bits: int) -> int:

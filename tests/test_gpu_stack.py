@@ -1,0 +1,104 @@
+"""GPU parity of the ResNet-18-shaped stack of encoded convolutions (W4A4) against the CPU oracle.
+
+The fp32 stem is glue, checked against a float64 convolution; from the stem's pooled output on,
+the oracle runs the same chain of encoded layers (range -> quantize -> integer convolution ->
+scale, residual add + max in fp32) and every layer must agree: int32 accumulators bit-exact,
+fp32 outputs within 1e-5 relative.  The small case is compared element by element through the
+whole chain; the full-size case (batch 128, 224 x 224) on sampled outputs of every layer, each
+computed by the oracle from the GPU's own input to that layer.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_1905_13389_b200 import inputs
+from paper_1905_13389_b200.resnet18 import BLOCKS, QuantResNet18Stack
+from tests._util import rel_close
+
+pytestmark = pytest.mark.gpu
+
+
+def test_stem_and_maxpool_against_float64(mpq, cuda):
+    x = inputs.config5_input(2, 70)                        # odd output size 35 -> ragged tiles
+    w = inputs.config5_weights()["conv1"]
+    y = mpq.stem_conv7x7(torch.from_numpy(x).to(cuda), torch.from_numpy(w).to(cuda), relu=False)
+    ref = torch.nn.functional.conv2d(torch.from_numpy(x).double(), torch.from_numpy(w).double(), stride=2, padding=3)
+    assert tuple(y.shape) == tuple(ref.shape) == (2, 64, 35, 35)
+    err = (y.cpu().double() - ref).abs().max().item()
+    assert err <= 1e-5 * ref.abs().max().item()            # 147-term fp32 sums against float64
+    yr = mpq.stem_conv7x7(torch.from_numpy(x).to(cuda), torch.from_numpy(w).to(cuda), relu=True)
+    assert torch.equal(yr, torch.clamp_min(y, 0))
+    p = mpq.maxpool3x3s2(yr)
+    assert torch.equal(p.cpu(), torch.nn.functional.max_pool2d(yr.cpu(), 3, 2, 1))
+
+
+def _oracle_block(x, ws, blk, stride, has_ds, a_bits, w_bits):
+    """One basic block on the CPU; returns {conv name: (acc, out)} and the block output."""
+    res = {}
+    acc1, t, _, _ = oracle.conv_layer(x, ws[blk + ".conv1"], a_bits, w_bits, stride, 1, True, oracle.HRELU)
+    res[blk + ".conv1"] = (acc1, t)
+    acc2, u, _, _ = oracle.conv_layer(t, ws[blk + ".conv2"], a_bits, w_bits, 1, 1, True, oracle.HRELU)
+    res[blk + ".conv2"] = (acc2, u)
+    if has_ds:
+        accd, sc, _, _ = oracle.conv_layer(x, ws[blk + ".downsample"], a_bits, w_bits, stride, 0, True, oracle.HRELU)
+        res[blk + ".downsample"] = (accd, sc)
+    else:
+        sc = x
+    return res, np.maximum(u + sc, np.float32(0))
+
+
+@pytest.mark.parametrize("a_bits,w_bits", [(4, 4), (2, 3)])
+def test_stack_small_chain_elementwise(mpq, cuda, a_bits, w_bits):
+    batch, size = 2, 64
+    ws = inputs.config5_weights()
+    x = inputs.config5_input(batch, size)
+    net = QuantResNet18Stack(ws, batch, size, a_bits, w_bits, cuda, keep_int32=True)
+    out = net.forward(torch.from_numpy(x).to(cuda))
+    torch.cuda.synchronize()
+    cur = net.pooled.cpu().numpy()                         # the oracle chain starts from the stem's output
+    assert cur.shape == (batch, 64, 16, 16) and cur.min() >= 0 and cur.max() > 0
+    for blk, _, _, stride, has_ds in BLOCKS:
+        res, cur = _oracle_block(cur, ws, blk, stride, has_ds, a_bits, w_bits)
+        for name, (acc, ref) in res.items():
+            assert np.array_equal(net.y_i32[name].cpu().numpy(), acc), name
+            assert rel_close(net.y[name].cpu().numpy(), ref), name
+        assert np.array_equal(net.block_out[blk].cpu().numpy(), cur), blk
+        assert np.unique(res[blk + ".conv2"][0]).size > 16
+    assert np.array_equal(out.cpu().numpy(), cur)
+
+
+def test_stack_full_size_sampled(mpq, cuda):
+    """Batch 128 at 224 x 224 in W4A4: every encoded layer, in the launch configuration that is
+    timed, on 40 sampled outputs (image corners and borders included) computed one by one."""
+    batch, size, a_bits, w_bits = 128, 224, 4, 4
+    ws = inputs.config5_weights()
+    net = QuantResNet18Stack(ws, batch, size, a_bits, w_bits, cuda, keep_int32=True)
+    net.forward(torch.from_numpy(inputs.config5_input(batch, size)).to(cuda))
+    torch.cuda.synchronize()
+    rng = np.random.default_rng(5)
+    layer_in = net.pooled
+    for blk, _, _, stride, has_ds in BLOCKS:
+        jobs = [(blk + ".conv1", layer_in), (blk + ".conv2", net.y[blk + ".conv1"])]
+        if has_ds:
+            jobs.append((blk + ".downsample", layer_in))
+        for name, xin in jobs:
+            conv = net.convs[name]
+            x = xin.cpu().numpy()
+            s_a = oracle.absmax(x, False, oracle.HRELU)
+            assert np.array_equal(net.x_scale[name if "downsample" not in name else blk + ".conv1"].cpu().numpy(), s_a)
+            s_w = oracle.absmax(ws[name], True)
+            qx = oracle.quantize(x, s_a, a_bits, act=oracle.HRELU)
+            qw = oracle.quantize(ws[name], s_w, w_bits, per_row=True)
+            yi = net.y_i32[name].cpu().numpy()
+            yf = net.y[name].cpu().numpy()
+            _, O, Ho, Wo = yi.shape
+            pts = [(0, 0, 0, 0), (batch - 1, O - 1, Ho - 1, Wo - 1), (1, 1, 0, Wo - 1), (2, O // 2, Ho - 1, 0)]
+            pts += [tuple(int(v) for v in (rng.integers(batch), rng.integers(O), rng.integers(Ho), rng.integers(Wo)))
+                    for _ in range(36)]
+            for (b, o, oh, ow) in pts:
+                acc = oracle.conv_at(qx, qw, conv.stride, conv.pad, b, o, oh, ow)
+                assert int(yi[b, o, oh, ow]) == acc, (name, b, o, oh, ow)
+                ref = oracle.scale(np.array([[acc]], np.int32), s_a[0], s_w[o:o + 1], a_bits, w_bits)[0, 0]
+                assert abs(float(yf[b, o, oh, ow]) - float(ref)) <= 1e-5 * abs(float(ref)), (name, b, o, oh, ow)
+        layer_in = net.block_out[blk]
