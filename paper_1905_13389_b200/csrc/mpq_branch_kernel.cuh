@@ -42,6 +42,8 @@ struct BranchParams {
     int N, C, H, W, O, KH, KW, stride, pad, Ho, Wo, Cw;
     int granule;               // words gathered per copy: 1 (C=32), 2 (C=64) or 4 (C % 128 == 0)
     const int32_t* tap_sums;   // [KH*KW][O]
+    uint32_t pow2[24];         // pow2[e] = 2^e: branch weights read from the constant bank, so that
+                               // "popcount * 2^e + acc" stays one integer multiply-add (FMA pipe)
 };
 
 __device__ __forceinline__ void cp_async_16(void* smem_dst, const void* gsrc, bool valid) {
@@ -59,9 +61,64 @@ __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commi
 template <int N>
 __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory"); }
 
-__device__ __forceinline__ int popc_xor4(const uint4& a, const uint4& b) {
-    return __popc(a.x ^ b.x) + __popc(a.y ^ b.y) + __popc(a.z ^ b.z) + __popc(a.w ^ b.w);
+// ---- The branch products of one output over one k-quad, with carry-save compression ---------
+// S += sum_{i,j} 2^(i+j) * popcount(h_i xor s_j) over the four words of a k-quad.  The 4*HB*SB
+// xor words are grouped by weight exponent e = i + j ("level").  Within a level three words of
+// equal weight are replaced by their bitwise sum (weight 2^e, one 3-input xor) and their bitwise
+// carry (weight 2^(e+1), one 3-input majority) -- a full adder on 32 bit positions at once, since
+// popc(a) + popc(b) + popc(c) = popc(a^b^c) + 2 popc(maj(a,b,c)).  Each such step trades one
+// population count (the narrow pipe of the SM: 16 lanes per clock) for two logic operations
+// (64 lanes per clock).  One round of disjoint triples per level leaves about half as many
+// population counts as xor words, which balances the two pipes; the weighted add of each count
+// is an integer multiply-add with 2^e taken from the constant bank, i.e. it runs on the FMA pipe.
+// All counts and array sizes are compile-time constants; the arrays live in registers.
+__host__ __device__ constexpr int pairs_at_level(int hb, int sb, int e) {
+    int n = 0;
+    for (int i = 0; i < hb; ++i) {
+        const int j = e - i;
+        if (j >= 0 && j < sb) ++n;
+    }
+    return n;
 }
+__device__ __forceinline__ uint32_t quad_word(const uint4& v, int c) {
+    return c == 0 ? v.x : c == 1 ? v.y : c == 2 ? v.z : v.w;
+}
+__device__ __forceinline__ uint32_t majority3(uint32_t a, uint32_t b, uint32_t c) { return (a & b) | (c & (a ^ b)); }
+
+template <int HB, int SB, int E, int NC, int ROUNDS>
+struct BranchLevel {
+    static constexpr int NF = 4 * pairs_at_level(HB, SB, E);   // fresh xor words of this level
+    static constexpr int N = NF + NC;                          // plus the carries of the level below
+    static constexpr int K = ROUNDS > 0 ? N / 3 : 0;           // full adders applied at this level
+    __device__ __forceinline__ static void run(const uint4 (&h)[HB], const uint4 (&s)[SB],
+                                               const uint32_t (&carry_in)[NC > 0 ? NC : 1],
+                                               uint32_t& acc, const BranchParams& p) {
+        if constexpr (N > 0) {
+            uint32_t w[N];
+#pragma unroll
+            for (int q = 0; q < NC; ++q) w[q] = carry_in[q];
+            int n = NC;
+#pragma unroll
+            for (int i = 0; i < HB; ++i) {
+                const int j = E - i;
+                if (j >= 0 && j < SB) {
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) w[n++] = quad_word(h[i], c) ^ quad_word(s[j], c);
+                }
+            }
+            uint32_t carry[K > 0 ? K : 1];
+#pragma unroll
+            for (int q = 0; q < K; ++q) {
+                const uint32_t a = w[3 * q], b = w[3 * q + 1], c = w[3 * q + 2];
+                carry[q] = majority3(a, b, c);
+                acc = (uint32_t)__popc(a ^ b ^ c) * p.pow2[E] + acc;
+            }
+#pragma unroll
+            for (int q = 3 * K; q < N; ++q) acc = (uint32_t)__popc(w[q]) * p.pow2[E] + acc;
+            BranchLevel<HB, SB, E + 1, K, ROUNDS>::run(h, s, carry, acc, p);
+        }
+    }
+};
 
 template <int HB, int SB>
 struct BranchTile {
@@ -69,6 +126,10 @@ struct BranchTile {
     static constexpr int KQ = (SB == 1) ? 8 : (SB == 2) ? 4 : (SB <= 4) ? 2 : 1;   // k-quads per stage
     static constexpr int STAGES = 3;
     static constexpr int THREADS = 256;
+    static constexpr int ROUNDS = 1;             // carry-save rounds per level (0 = plain xor + popcount)
+    // the k-quads of a stage are unrolled only while the loop body stays small enough for the
+    // instruction cache (about 12 instructions per plane pair per output)
+    static constexpr bool UNROLL_KQ = HB * SB <= 4;
 };
 
 template <int HB, int SB, int TS, int MODE>
@@ -184,8 +245,7 @@ branch_kernel(const BranchParams p) {
         }
         const uint4* hs = smem + (size_t)(it % STAGES) * STAGE_QUADS;
         const uint4* ss = hs + H_QUADS;
-#pragma unroll
-        for (int kq = 0; kq < KQ; ++kq) {
+        auto one_quad = [&](int kq) {
             uint4 h[TH][HB];
 #pragma unroll
             for (int a = 0; a < TH; ++a)
@@ -193,16 +253,21 @@ branch_kernel(const BranchParams p) {
                 for (int i = 0; i < HB; ++i) h[a][i] = hs[(i * KQ + kq) * BH + ty + 16 * a];
 #pragma unroll
             for (int b = 0; b < TS; ++b) {
+                uint4 s[SB];
 #pragma unroll
-                for (int j = 0; j < SB; ++j) {
-                    const uint4 s = ss[(j * KQ + kq) * BS + tx + 16 * b];
+                for (int j = 0; j < SB; ++j) s[j] = ss[(j * KQ + kq) * BS + tx + 16 * b];
+                const uint32_t none[1] = {0u};
 #pragma unroll
-                    for (int a = 0; a < TH; ++a)
-#pragma unroll
-                        for (int i = 0; i < HB; ++i)
-                            acc[a][b] += (uint32_t)popc_xor4(h[a][i], s) << (i + j);
-                }
+                for (int a = 0; a < TH; ++a)
+                    BranchLevel<HB, SB, 0, 0, T::ROUNDS>::run(h[a], s, none, acc[a][b], p);
             }
+        };
+        if (T::UNROLL_KQ) {
+#pragma unroll
+            for (int kq = 0; kq < KQ; ++kq) one_quad(kq);
+        } else {
+#pragma unroll 1
+            for (int kq = 0; kq < KQ; ++kq) one_quad(kq);
         }
     }
     cp_async_wait<0>();

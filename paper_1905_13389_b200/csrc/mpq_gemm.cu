@@ -34,6 +34,10 @@ static int dispatch_conv(int hb, int sb, const BranchParams& p, cudaStream_t st)
     return MPQ_ERR_UNSUPPORTED;
 }
 
+static void fill_pow2(BranchParams& p) {
+    for (int e = 0; e < 24; ++e) p.pow2[e] = 1u << e;
+}
+
 // k * L_a * L_w must stay below 2^31 so that every |acc| fits int32.
 static bool int32_headroom(int64_t k, int a_bits, int w_bits) {
     const int64_t LL = (int64_t)((1 << a_bits) - 1) * ((1 << w_bits) - 1);
@@ -61,6 +65,7 @@ extern "C" int mpq_gemm(const uint32_t* a_planes, int a_bits, const uint32_t* b_
     p.rw = row_words(k); p.k = k;
     p.out_i32 = c_i32; p.out_f32 = c_f32; p.ldc = ldc;
     p.a_scale = a_scale; p.w_scale = b_scale; p.w_per_row = b_mode == MPQ_SCALE_PER_ROW;
+    fill_pow2(p);
     return dispatch_gemm(a_bits, b_bits, p, (cudaStream_t)stream);
 }
 
@@ -92,6 +97,7 @@ extern "C" int mpq_conv(const uint32_t* x_planes, int a_bits, int N, int C, int 
     p.N = N; p.C = C; p.H = H; p.W = W; p.O = O; p.KH = KH; p.KW = KW; p.stride = stride; p.pad = pad;
     p.Cw = C / 32; p.granule = p.Cw >= 4 ? 4 : p.Cw;
     p.tap_sums = tap_sums;
+    fill_pow2(p);
     // held = weights (w_bits planes), streamed = activations (a_bits planes)
     return dispatch_conv(w_bits, a_bits, p, (cudaStream_t)stream);
 }
