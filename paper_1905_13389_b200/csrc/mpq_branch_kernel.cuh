@@ -68,7 +68,7 @@ __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_gr
 // carry (weight 2^(e+1), one 3-input majority) -- a full adder on 32 bit positions at once, since
 // popc(a) + popc(b) + popc(c) = popc(a^b^c) + 2 popc(maj(a,b,c)).  Each such step trades one
 // population count (the narrow pipe of the SM: 16 lanes per clock) for two logic operations
-// (64 lanes per clock).  One round of disjoint triples per level leaves about half as many
+// (64 lanes per clock).  Spending about one adder per two xor words leaves half as many
 // population counts as xor words, which balances the two pipes; the weighted add of each count
 // is an integer multiply-add with 2^e taken from the constant bank, i.e. it runs on the FMA pipe.
 // All counts and array sizes are compile-time constants; the arrays live in registers.
@@ -83,13 +83,62 @@ __host__ __device__ constexpr int pairs_at_level(int hb, int sb, int e) {
 __device__ __forceinline__ uint32_t quad_word(const uint4& v, int c) {
     return c == 0 ? v.x : c == 1 ? v.y : c == 2 ? v.z : v.w;
 }
-__device__ __forceinline__ uint32_t majority3(uint32_t a, uint32_t b, uint32_t c) { return (a & b) | (c & (a ^ b)); }
+// Full adder on 32 bit positions: each half is exactly one 3-input logic operation (written as
+// lop3 with its truth table so that the compiler cannot split it into 2-input steps).
+__device__ __forceinline__ uint32_t majority3(uint32_t a, uint32_t b, uint32_t c) {
+    uint32_t d;
+    asm("lop3.b32 %0, %1, %2, %3, 0xE8;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+    return d;
+}
+__device__ __forceinline__ uint32_t parity3(uint32_t a, uint32_t b, uint32_t c) {
+    uint32_t d;
+    asm("lop3.b32 %0, %1, %2, %3, 0x96;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+    return d;
+}
 
-template <int HB, int SB, int E, int NC, int ROUNDS>
+// One level's working set: up to BUDGET full adders, applied in rounds of disjoint triples
+// (independent of one another, so they pipeline); what is left after the last round is counted.
+template <int N, int BUDGET>
+struct CarrySave {
+    static constexpr int K = (N / 3 < BUDGET) ? N / 3 : BUDGET;            // adders of this round
+    static constexpr int REST = N - 2 * K;                                  // words after the round
+    static constexpr int TOTAL = K == 0 ? 0 : K + CarrySave<(K == 0 ? 0 : REST), (K == 0 ? 0 : BUDGET - K)>::TOTAL;
+    // w: the N words; carry[at ...] receives the TOTAL carries; the counts go to acc with `weight`
+    template <int NCARRY>
+    __device__ __forceinline__ static void run(const uint32_t (&w)[N > 0 ? N : 1], uint32_t (&carry)[NCARRY], int at,
+                                               uint32_t& acc, uint32_t weight) {
+        if constexpr (K == 0) {
+#pragma unroll
+            for (int q = 0; q < N; ++q) acc = (uint32_t)__popc(w[q]) * weight + acc;
+        } else {
+            uint32_t r[REST];
+#pragma unroll
+            for (int q = 0; q < K; ++q) {
+                const uint32_t a = w[3 * q], b = w[3 * q + 1], c = w[3 * q + 2];
+                carry[at + q] = majority3(a, b, c);
+                r[q] = parity3(a, b, c);
+            }
+#pragma unroll
+            for (int q = 3 * K; q < N; ++q) r[K + q - 3 * K] = w[q];
+            CarrySave<REST, BUDGET - K>::run(r, carry, at + K, acc, weight);
+        }
+    }
+};
+template <>
+struct CarrySave<0, 0> {
+    static constexpr int TOTAL = 0;
+    template <int NCARRY>
+    __device__ __forceinline__ static void run(const uint32_t (&)[1], uint32_t (&)[NCARRY], int, uint32_t&, uint32_t) {}
+};
+
+// Level E of one output: NC carries from the level below plus the fresh xor words; BUDGET is the
+// number of full adders still to be spent on this and the higher levels (lower levels first).
+template <int HB, int SB, int E, int NC, int BUDGET>
 struct BranchLevel {
     static constexpr int NF = 4 * pairs_at_level(HB, SB, E);   // fresh xor words of this level
-    static constexpr int N = NF + NC;                          // plus the carries of the level below
-    static constexpr int K = ROUNDS > 0 ? N / 3 : 0;           // full adders applied at this level
+    static constexpr int N = NF + NC;
+    using CS = CarrySave<N, (N >= 3 ? BUDGET : 0)>;
+    static constexpr int K = CS::TOTAL;
     __device__ __forceinline__ static void run(const uint4 (&h)[HB], const uint4 (&s)[SB],
                                                const uint32_t (&carry_in)[NC > 0 ? NC : 1],
                                                uint32_t& acc, const BranchParams& p) {
@@ -107,15 +156,8 @@ struct BranchLevel {
                 }
             }
             uint32_t carry[K > 0 ? K : 1];
-#pragma unroll
-            for (int q = 0; q < K; ++q) {
-                const uint32_t a = w[3 * q], b = w[3 * q + 1], c = w[3 * q + 2];
-                carry[q] = majority3(a, b, c);
-                acc = (uint32_t)__popc(a ^ b ^ c) * p.pow2[E] + acc;
-            }
-#pragma unroll
-            for (int q = 3 * K; q < N; ++q) acc = (uint32_t)__popc(w[q]) * p.pow2[E] + acc;
-            BranchLevel<HB, SB, E + 1, K, ROUNDS>::run(h, s, carry, acc, p);
+            CS::run(w, carry, 0, acc, p.pow2[E]);
+            BranchLevel<HB, SB, E + 1, K, BUDGET - K>::run(h, s, carry, acc, p);
         }
     }
 };
@@ -126,7 +168,9 @@ struct BranchTile {
     static constexpr int KQ = (SB == 1) ? 8 : (SB == 2) ? 4 : (SB <= 4) ? 2 : 1;   // k-quads per stage
     static constexpr int STAGES = 3;
     static constexpr int THREADS = 256;
-    static constexpr int ROUNDS = 1;             // carry-save rounds per level (0 = plain xor + popcount)
+    // full adders per output and k-quad: half of the 4*HB*SB xor words balances the two pipes
+    // (each adder costs two logic operations and saves one population count)
+    static constexpr int CSA_BUDGET = 2 * HB * SB;
     // the k-quads of a stage are unrolled only while the loop body stays small enough for the
     // instruction cache (about 12 instructions per plane pair per output)
     static constexpr bool UNROLL_KQ = HB * SB <= 4;
@@ -259,7 +303,7 @@ branch_kernel(const BranchParams p) {
                 const uint32_t none[1] = {0u};
 #pragma unroll
                 for (int a = 0; a < TH; ++a)
-                    BranchLevel<HB, SB, 0, 0, T::ROUNDS>::run(h[a], s, none, acc[a][b], p);
+                    BranchLevel<HB, SB, 0, 0, T::CSA_BUDGET>::run(h[a], s, none, acc[a][b], p);
             }
         };
         if (T::UNROLL_KQ) {
