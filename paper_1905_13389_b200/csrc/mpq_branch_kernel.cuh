@@ -306,12 +306,15 @@ branch_kernel(const BranchParams p) {
                     BranchLevel<HB, SB, 0, 0, T::CSA_BUDGET>::run(h[a], s, none, acc[a][b], p);
             }
         };
+        // the last stage may hold fewer than KQ k-quads of data: skip the rest (they are all zero)
+        const int kq_live = (int)min((int64_t)KQ, kq_total - (int64_t)it * KQ);
         if (T::UNROLL_KQ) {
 #pragma unroll
-            for (int kq = 0; kq < KQ; ++kq) one_quad(kq);
+            for (int kq = 0; kq < KQ; ++kq)
+                if (kq < kq_live) one_quad(kq);
         } else {
 #pragma unroll 1
-            for (int kq = 0; kq < KQ; ++kq) one_quad(kq);
+            for (int kq = 0; kq < kq_live; ++kq) one_quad(kq);
         }
     }
     cp_async_wait<0>();
