@@ -1,0 +1,206 @@
+"""Per-workload measurements behind ``bench.py --full FILE``: the five synthetic workloads
+(single small GEMM, fully-connected layer, 3x3 convolution, bit-width sweep, ResNet-18-shaped
+stack) and the encoders, each timed with CUDA events on the launching stream after warm-up.
+Everything goes through the C ABI binding; nothing here touches the CPU oracle."""
+from __future__ import annotations
+
+import json
+import statistics
+
+import numpy as np
+import torch
+
+from paper_1905_13389_b200 import binding as mpq
+from paper_1905_13389_b200 import inputs
+from paper_1905_13389_b200.resnet18 import QuantResNet18Stack
+
+
+def _events_ms(fn, iters=20, warmup=5):
+    for _ in range(warmup):
+        fn()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(iters):
+        fn()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / iters
+
+
+def _graph_ms(fn, iters=20, warmup=5):
+    """Short kernels: replay `iters` launches from one CUDA graph so that host launch cost
+    (ctypes marshalling, ~10 us per call) does not sit between the kernels being timed."""
+    for _ in range(warmup):
+        fn()
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    st = torch.cuda.Stream()
+    with torch.cuda.stream(st):
+        with torch.cuda.graph(g, stream=st):
+            for _ in range(iters):
+                fn()
+    g.replay()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    g.replay()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / iters
+
+
+def run_suite(dev: torch.device, hbm_gbs: float, path: str):
+    up = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(dev)
+    popc_peak, mhz, sms = mpq.measure_popc_peak()
+    mix, _, _ = mpq.measure_mix_peak(4)
+    branch_peak = 2.0 * mix
+    out = {"popc_peak_gpopc_s": popc_peak / 1e9, "branch_peak_gpopc_s": branch_peak / 1e9, "probe_sm_mhz": mhz,
+           "hbm_gbs": hbm_gbs}
+
+    def product_record(ms, m, n, k, a_bits, w_bits, popcs):
+        return {"ms": ms, "equivalent_tops": 2.0 * m * n * k / (ms * 1e-3) / 1e12,
+                "binary_tops": 2.0 * m * n * k * a_bits * w_bits / (ms * 1e-3) / 1e12,
+                "gpopc_s": popcs / (ms * 1e-3) / 1e9, "frac_of_branch_peak": popcs / (ms * 1e-3) / branch_peak,
+                "frac_of_plain_popc_peak": popcs / (ms * 1e-3) / popc_peak}
+
+    # ---- workload 1: one small GEMM (launch-latency bound) --------------------------------------
+    c = inputs.config1()
+    x, w = up(c["x"]), up(c["w"])
+    sa, sw = mpq.absmax(x, 0, mpq.ACT_HRELU), mpq.absmax(w)
+    ap, wp = mpq.encode(x, sa, 2, 0, mpq.ACT_HRELU), mpq.encode(w, sw, 2)
+    ci = torch.empty((64, 64), dtype=torch.int32, device=dev)
+    cf = torch.empty((64, 64), dtype=torch.float32, device=dev)
+    ms = _graph_ms(lambda: mpq.gemm(ap, 2, wp, 2, 64, 64, 512, ci, cf, sa, sw), 50)
+    out["gemm_w2a2_64x64x512"] = {"us": ms * 1e3}
+
+    # ---- workload 4: the bit-width sweep at 4096^3 ----------------------------------------------
+    size = 4096
+    c4 = inputs.config4(2, 2, size)
+    x, w = up(c4["x"]), up(c4["w"])
+    sa, sw = mpq.absmax(x, 0, mpq.ACT_HRELU), mpq.absmax(w)
+    ci = torch.empty((size, size), dtype=torch.int32, device=dev)
+    sweep = {}
+    for (w_bits, a_bits) in inputs.SWEEP_BITS:
+        ap, wp = mpq.encode(x, sa, a_bits, 0, mpq.ACT_HRELU), mpq.encode(w, sw, w_bits)
+        ms = _events_ms(lambda: mpq.gemm(ap, a_bits, wp, w_bits, size, size, size, ci, None), 10, 3)
+        sweep["w%da%d" % (w_bits, a_bits)] = product_record(ms, size, size, size, a_bits, w_bits,
+                                                             float(a_bits * w_bits) * size * size * (size // 32))
+    out["gemm_sweep_4096"] = sweep
+
+    # ---- encoders on the sweep's operands (64 MiB fp32 each; four buffers in rotation) ----------
+    xs = [x, w, torch.randn_like(x), torch.randn_like(x)]
+    enc = {}
+    for bits in (1, 2, 3, 4, 8):
+        planes = torch.empty((bits, size, mpq.row_words(size)), dtype=torch.int32, device=dev)
+        i = [0]
+
+        def f():
+            mpq.encode(xs[i[0] % 4], sa, bits, 0, mpq.ACT_HTANH, out=planes)
+            i[0] += 1
+        ms = _graph_ms(f)
+        by = size * size * (4 + bits / 8.0)
+        enc["rows_4096x4096_b%d" % bits] = {"us": ms * 1e3, "gb_s": by / (ms * 1e-3) / 1e9,
+                                            "frac_of_hbm": by / (ms * 1e-3) / 1e9 / hbm_gbs}
+    i = [0]
+    s1 = torch.empty(1, dtype=torch.float32, device=dev)
+
+    def f():
+        mpq.absmax(xs[i[0] % 4], out=s1)
+        i[0] += 1
+    ms = _graph_ms(f)
+    enc["absmax_4096x4096"] = {"us": ms * 1e3, "gb_s": size * size * 4 / (ms * 1e-3) / 1e9,
+                               "frac_of_hbm": size * size * 4 / (ms * 1e-3) / 1e9 / hbm_gbs}
+    del xs, x, w
+
+    # ---- workload 2: fully-connected layer W2A2 --------------------------------------------------
+    c = inputs.config2()
+    x, w = up(c["x"]), up(c["w"])
+    m, n, k = c["m"], c["n"], c["k"]
+    sa, sw = mpq.absmax(x, 0, mpq.ACT_HRELU), mpq.absmax(w, mpq.SCALE_PER_ROW)
+    ap = mpq.encode(x, sa, 2, 0, mpq.ACT_HRELU)
+    wp = torch.empty((2, n, mpq.row_words(k)), dtype=torch.int32, device=dev)
+    w2 = w.clone()
+    i = [0]
+
+    def f():
+        mpq.encode(w if i[0] % 2 == 0 else w2, sw, 2, mpq.SCALE_PER_ROW, out=wp)
+        i[0] += 1
+    ms_we = _graph_ms(f)
+    by = n * k * 4.25
+    cf = torch.empty((m, n), dtype=torch.float32, device=dev)
+    ms = _graph_ms(lambda: mpq.gemm(ap, 2, wp, 2, m, n, k, None, cf, sa, sw, mpq.SCALE_PER_ROW))
+    rec = product_record(ms, m, n, k, 2, 2, 4.0 * m * n * (k // 32))
+    rec["weight_encode"] = {"us": ms_we * 1e3, "gb_s": by / (ms_we * 1e-3) / 1e9,
+                            "frac_of_hbm": by / (ms_we * 1e-3) / 1e9 / hbm_gbs}
+    enc["rows_4096x9216_b2_per_row_scale"] = rec["weight_encode"]
+    out["fc_w2a2_64x4096x9216"] = rec
+    del w, w2
+
+    # ---- workload 3: 3x3 convolution W3A3 --------------------------------------------------------
+    c = inputs.config3()
+    x, w = up(c["x"]), up(c["w"])
+    N, C, H, W = x.shape
+    O = w.shape[0]
+    sa, sw = mpq.absmax(x, 0, mpq.ACT_HRELU), mpq.absmax(w, mpq.SCALE_PER_ROW)
+    xp = mpq.encode_nchw(x, sa, 3, mpq.ACT_HRELU)
+    wpl, taps = mpq.encode_oihw(w, sw, 3, mpq.SCALE_PER_ROW)
+    yf = torch.empty((N, O, H, W), dtype=torch.float32, device=dev)
+    ms = _graph_ms(lambda: mpq.conv(xp, 3, N, C, H, W, wpl, 3, taps, O, 3, 3, 1, 1, None, yf, sa, sw, mpq.SCALE_PER_ROW))
+    M, K = N * H * W, 9 * C
+    out["conv3x3_w3a3_32x256x14x14"] = product_record(ms, M, O, K, 3, 3, 9.0 * M * O * (K // 32))
+    ms = _graph_ms(lambda: mpq.encode_nchw(x, sa, 3, mpq.ACT_HRELU, out=xp))
+    out["conv3x3_w3a3_32x256x14x14"]["encode_nchw_us"] = ms * 1e3
+
+    # ---- workload 5: ResNet-18-shaped stack, W4A4, batch 128 -------------------------------------
+    batch = 128
+    net = QuantResNet18Stack(inputs.config5_weights(), batch, 224, 4, 4, dev)
+    x = up(inputs.config5_input(batch, 224))
+    for _ in range(3):
+        net.forward(x)
+    torch.cuda.synchronize()
+    steps, evs = 5, []
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        ev = {}
+        net.forward(x, ev)
+        evs.append(ev)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    layers = {}
+    quant_ms = 0.0
+    for name in evs[0]:
+        t = statistics.mean(ev[name][0].elapsed_time(ev[name][1]) for ev in evs)
+        rec = {"ms": t}
+        if name in net.convs:
+            cv = net.convs[name]
+            Cc, Hh, Ww = net.in_shape[name]
+            Ho, Wo = cv.out_hw(Hh, Ww)
+            popcs = 16.0 * batch * Ho * Wo * cv.O * (cv.KH * cv.KW * Cc // 32)
+            rec.update({"span": "range + encode + conv" if "downsample" not in name else "conv",
+                        "frac_of_branch_peak": popcs / (t * 1e-3) / branch_peak,
+                        "frac_of_plain_popc_peak": popcs / (t * 1e-3) / popc_peak})
+            quant_ms += t
+        layers[name] = rec
+    out["resnet18_stack_w4a4_b128"] = {"ms_per_step": ms, "images_per_s": batch / (ms * 1e-3),
+                                       "quantized_layers_ms": quant_ms, "layers": layers}
+    # activation encoder of the first stage (NCHW variant, 102.8 MB in)
+    xin = net.pooled
+    i = [0]
+    alt = torch.relu(torch.randn_like(xin))
+    s_in = mpq.absmax(xin, 0, mpq.ACT_HRELU)
+    pl = net.x_planes["layer1.0.conv1"]
+
+    def f():
+        mpq.encode_nchw(xin if i[0] % 2 == 0 else alt, s_in, 4, mpq.ACT_HRELU, out=pl)
+        i[0] += 1
+    ms = _graph_ms(f)
+    by = xin.numel() * 4.5
+    enc["nchw_128x64x56x56_b4"] = {"us": ms * 1e3, "gb_s": by / (ms * 1e-3) / 1e9,
+                                   "frac_of_hbm": by / (ms * 1e-3) / 1e9 / hbm_gbs}
+    out["encoders"] = enc
+    with open(path, "w") as fh:
+        json.dump(out, fh, indent=1)
+    return out

@@ -186,6 +186,14 @@ int mpq_linear_host(const float* x_host, const float* w_host, int64_t m, int64_t
  * observed inside the kernel; sms: multiprocessor count.  Any pointer may be NULL. */
 int mpq_measure_popc_peak(double* popc_per_s, double* sm_mhz, int* sms, void* stream);
 
+/* ---- Roofline denominator of the carry-save form of the branch products (Eq. 7-10 computed
+ * with full adders on the xor words): issue rate of a register-only loop whose groups hold
+ * `logic_per_popc` (0..8) three-input logic operations, one population count and one integer
+ * multiply-add.  With one full adder per two xor words the kernel's mix is 4 logic operations
+ * per population count and one group stands for two algorithmic word-popcounts.  Synchronous.
+ * groups_per_s: lane-level groups per second over the whole chip. */
+int mpq_measure_mix_peak(int logic_per_popc, double* groups_per_s, double* sm_mhz, int* sms, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -63,6 +63,9 @@ def lib() -> ctypes.CDLL:
         L.mpq_linear_host.argtypes = [P, P, i64, i64, i64, i32, i32, i32, i32, P, P, P, i64, P]
         L.mpq_measure_popc_peak.argtypes = [ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double),
                                             ctypes.POINTER(ctypes.c_int), P]
+        L.mpq_measure_mix_peak.argtypes = [i32, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double),
+                                           ctypes.POINTER(ctypes.c_int), P]
+        L.mpq_measure_mix_peak.restype = i32
         for name in ("mpq_absmax", "mpq_encode", "mpq_encode_nchw", "mpq_encode_oihw", "mpq_gemm", "mpq_conv",
                      "mpq_add_relu", "mpq_stem_conv7x7", "mpq_maxpool3x3s2", "mpq_linear", "mpq_linear_static", "mpq_linear_host", "mpq_measure_popc_peak"):
             getattr(L, name).restype = i32
@@ -270,4 +273,12 @@ def measure_popc_peak():
     rate, mhz, sms = ctypes.c_double(), ctypes.c_double(), ctypes.c_int()
     _check(lib().mpq_measure_popc_peak(ctypes.byref(rate), ctypes.byref(mhz), ctypes.byref(sms), _stream()),
            "mpq_measure_popc_peak")
+    return rate.value, mhz.value, sms.value
+
+
+def measure_mix_peak(logic_per_popc: int = 4):
+    """(groups per second of `logic_per_popc` logic ops + 1 POPC + 1 multiply-add, SM MHz, SM count)."""
+    rate, mhz, sms = ctypes.c_double(), ctypes.c_double(), ctypes.c_int()
+    _check(lib().mpq_measure_mix_peak(logic_per_popc, ctypes.byref(rate), ctypes.byref(mhz), ctypes.byref(sms),
+                                      _stream()), "mpq_measure_mix_peak")
     return rate.value, mhz.value, sms.value
