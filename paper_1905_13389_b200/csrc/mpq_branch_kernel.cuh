@@ -41,6 +41,9 @@ struct BranchParams {
     // CONV only
     int N, C, H, W, O, KH, KW, stride, pad, Ho, Wo, Cw;
     int granule;               // words gathered per copy: 1 (C=32), 2 (C=64) or 4 (C % 128 == 0)
+    int granule_shift;         // log2(4 / granule): copies per k-quad
+    int tap_granules;          // copies per filter tap = Cw / granule
+    uint32_t tap_magic;        // ceil(2^32 / tap_granules): copy index / tap_granules by one multiply
     const int32_t* tap_sums;   // [KH*KW][O]
     uint32_t pow2[24];         // pow2[e] = 2^e: branch weights read from the constant bank, so that
                                // "popcount * 2^e + acc" stays one integer multiply-add (FMA pipe)
@@ -190,6 +193,7 @@ branch_kernel(const BranchParams p) {
     __shared__ int row_n[MODE == kModeConv ? BS : 1];      // image index, or -1 for rows past the end
     __shared__ int row_ih0[MODE == kModeConv ? BS : 1];    // top-left input coordinate of the window
     __shared__ int row_iw0[MODE == kModeConv ? BS : 1];
+    __shared__ int row_pix[MODE == kModeConv ? BS : 1];    // (n*H + ih0)*W + iw0: pixel index of the window origin
 
     const int tid = threadIdx.x;
     const int tx = tid & 15, ty = tid >> 4;
@@ -209,8 +213,9 @@ branch_kernel(const BranchParams p) {
                 row_n[r] = n;
                 row_ih0[r] = (rem / p.Wo) * p.stride - p.pad;
                 row_iw0[r] = (rem % p.Wo) * p.stride - p.pad;
+                row_pix[r] = (n * p.H + row_ih0[r]) * p.W + row_iw0[r];
             } else {
-                row_n[r] = -1; row_ih0[r] = 0; row_iw0[r] = 0;
+                row_n[r] = -1; row_ih0[r] = -(1 << 20); row_iw0[r] = 0; row_pix[r] = 0;   // never inside the image
             }
         }
         __syncthreads();
@@ -244,21 +249,25 @@ branch_kernel(const BranchParams p) {
                 }
             }
         } else {
-            // implicit im2col: one copy = `granule` words of one tap of one pixel (never crosses a tap)
+            // implicit im2col: one copy = `granule` words of one tap of one pixel (never crosses a tap).
+            // Index arithmetic is kept to shifts, compile-time divisors and one multiply-high.
             const int G = p.granule;
-            const int parts = 4 / G;
-            const int granules = S_QUADS * parts;
-            const int taps = p.KH * p.KW;
+            const int gs = p.granule_shift;                 // copies per k-quad = 1 << gs
+            const int granules = S_QUADS << gs;
+            const int64_t plane_words = (int64_t)p.N * p.H * p.W * p.Cw;
             for (int id = tid; id < granules; id += 256) {
-                const int part = id % parts, kq = (id / parts) % KQ;
-                const int row = (id / (parts * KQ)) % BS, plane = id / (parts * KQ * BS);
-                const int64_t kword = (kq0 + kq) * 4 + part * G;
-                const int tap = (int)(kword / p.Cw), cw = (int)(kword % p.Cw);
-                const int n = row_n[row];
-                const int ih = row_ih0[row] + tap / p.KW, iw = row_iw0[row] + tap % p.KW;
-                const bool ok = n >= 0 && tap < taps && ih >= 0 && ih < p.H && iw >= 0 && iw < p.W;
-                const uint32_t* src = ok ? p.streamed + ((((int64_t)plane * p.N + n) * p.H + ih) * p.W + iw) * p.Cw + cw
-                                         : p.streamed;
+                const int part = id & ((1 << gs) - 1);
+                const int q = id >> gs;
+                const int kq = q % KQ, row = (q / KQ) % BS, plane = q / (KQ * BS);
+                const uint32_t copy = (uint32_t)(((kq0 + kq) << gs) + part);   // copy index along k
+                const uint32_t tap = p.tap_granules == 1 ? copy : __umulhi(copy, p.tap_magic);
+                const int cw = (int)(copy - tap * p.tap_granules) * G;
+                const int kh = p.KW == 1 ? 0 : (int)((tap * 11u) >> 5);         // tap / 3 for tap < 9
+                const int kw = (int)tap - kh * p.KW;
+                const int ih = row_ih0[row] + kh, iw = row_iw0[row] + kw;
+                const bool ok = tap < (uint32_t)(p.KH * p.KW) && ih >= 0 && ih < p.H && iw >= 0 && iw < p.W;
+                const int pixel = row_pix[row] + kh * p.W + kw;
+                const uint32_t* src = ok ? p.streamed + plane * plane_words + (int64_t)pixel * p.Cw + cw : p.streamed;
                 uint32_t* dst = reinterpret_cast<uint32_t*>(ss + (plane * KQ + kq) * BS + row) + part * G;
                 if (G == 4) cp_async_16(dst, src, ok);
                 else if (G == 2) cp_async_small<8>(dst, src, ok);
@@ -413,14 +422,27 @@ static int launch_branch(const BranchParams& p, cudaStream_t st) {
     return launch_status();
 }
 
-// Streamed-side tile width: 128 columns normally, 32 when the wide tile would leave most of the
-// 148 SMs idle (skinny problems such as a batch-64 fully-connected layer).
-template <int HB, int SB>
-static int launch_gemm_auto(const BranchParams& p, cudaStream_t st) {
+// Streamed-side tile width (16*TS items): the widest tile has the least shared-memory traffic per
+// population count, but a grid of few large tiles leaves SMs idle in its last wave.  Pick the
+// width with the smallest estimated makespan: waves of (2 CTAs x 148 SMs) tiles, each costing
+// its width times a measured per-width inefficiency.
+template <int HB, int SB, int MODE>
+static int launch_auto(const BranchParams& p, cudaStream_t st) {
     using T = BranchTile<HB, SB>;
-    const int64_t wide = ceil_div(p.streamed_rows, 128) * ceil_div(p.held_rows, 16 * T::TH);
-    if (wide >= 148) return launch_branch<HB, SB, 8, kModeGemm>(p, st);
-    return launch_branch<HB, SB, 2, kModeGemm>(p, st);
+    const int64_t held_tiles = ceil_div(p.held_rows, 16 * T::TH);
+    const int64_t slots = 2 * 148;
+    const double penalty[3] = {1.00, 1.05, 1.20};      // TS = 8, 4, 2
+    int best = 0;
+    double best_cost = 0.0;
+    for (int c = 0; c < 3; ++c) {
+        const int ts = 8 >> c;
+        const int64_t tiles = ceil_div(p.streamed_rows, 16 * ts) * held_tiles;
+        const double cost = (double)ceil_div(tiles, slots) * ts * penalty[c];
+        if (c == 0 || cost < best_cost) { best = c; best_cost = cost; }
+    }
+    if (best == 0) return launch_branch<HB, SB, 8, MODE>(p, st);
+    if (best == 1) return launch_branch<HB, SB, 4, MODE>(p, st);
+    return launch_branch<HB, SB, 2, MODE>(p, st);
 }
 
 // One translation unit per held-operand width instantiates all eight streamed widths.

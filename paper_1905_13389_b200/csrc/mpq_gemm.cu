@@ -96,6 +96,11 @@ extern "C" int mpq_conv(const uint32_t* x_planes, int a_bits, int N, int C, int 
     p.a_scale = x_scale; p.w_scale = w_scale; p.w_per_row = w_mode == MPQ_SCALE_PER_ROW;
     p.N = N; p.C = C; p.H = H; p.W = W; p.O = O; p.KH = KH; p.KW = KW; p.stride = stride; p.pad = pad;
     p.Cw = C / 32; p.granule = p.Cw >= 4 ? 4 : p.Cw;
+    p.granule_shift = p.granule == 4 ? 0 : p.granule == 2 ? 1 : 2;
+    p.tap_granules = p.Cw / p.granule;
+    p.tap_magic = p.tap_granules > 1 ? (uint32_t)((((uint64_t)1 << 32) + p.tap_granules - 1) / p.tap_granules) : 0u;
+    // the gather indexes pixels with 32-bit integers and divides copy indices below 2^16 exactly
+    if ((int64_t)N * H * W >= ((int64_t)1 << 31) || (p.rw << p.granule_shift) >= 65536) return MPQ_ERR_UNSUPPORTED;
     p.tap_sums = tap_sums;
     fill_pow2(p);
     // held = weights (w_bits planes), streamed = activations (a_bits planes)
