@@ -134,15 +134,16 @@ struct CarrySave<0, 0> {
     __device__ __forceinline__ static void run(const uint32_t (&)[1], uint32_t (&)[NCARRY], int, uint32_t&, uint32_t) {}
 };
 
-// Level E of one output: NC carries from the level below plus the fresh xor words; BUDGET is the
-// number of full adders still to be spent on this and the higher levels (lower levels first).
-template <int HB, int SB, int E, int NC, int BUDGET>
+// Level E of one output: NC carries from the level below plus the fresh xor words of GQ k-quads;
+// BUDGET is the number of full adders still to be spent on this and the higher levels (lower
+// levels first).  h and s hold the planes of the GQ k-quads, quad-major: h[g * HB + i].
+template <int HB, int SB, int GQ, int E, int NC, int BUDGET>
 struct BranchLevel {
-    static constexpr int NF = 4 * pairs_at_level(HB, SB, E);   // fresh xor words of this level
+    static constexpr int NF = 4 * GQ * pairs_at_level(HB, SB, E);   // fresh xor words of this level
     static constexpr int N = NF + NC;
     using CS = CarrySave<N, (N >= 3 ? BUDGET : 0)>;
     static constexpr int K = CS::TOTAL;
-    __device__ __forceinline__ static void run(const uint4 (&h)[HB], const uint4 (&s)[SB],
+    __device__ __forceinline__ static void run(const uint4 (&h)[GQ * HB], const uint4 (&s)[GQ * SB],
                                                const uint32_t (&carry_in)[NC > 0 ? NC : 1],
                                                uint32_t& acc, const BranchParams& p) {
         if constexpr (N > 0) {
@@ -151,29 +152,35 @@ struct BranchLevel {
             for (int q = 0; q < NC; ++q) w[q] = carry_in[q];
             int n = NC;
 #pragma unroll
-            for (int i = 0; i < HB; ++i) {
-                const int j = E - i;
-                if (j >= 0 && j < SB) {
+            for (int g = 0; g < GQ; ++g) {
 #pragma unroll
-                    for (int c = 0; c < 4; ++c) w[n++] = quad_word(h[i], c) ^ quad_word(s[j], c);
+                for (int i = 0; i < HB; ++i) {
+                    const int j = E - i;
+                    if (j >= 0 && j < SB) {
+#pragma unroll
+                        for (int c = 0; c < 4; ++c) w[n++] = quad_word(h[g * HB + i], c) ^ quad_word(s[g * SB + j], c);
+                    }
                 }
             }
             uint32_t carry[K > 0 ? K : 1];
             CS::run(w, carry, 0, acc, p.pow2[E]);
-            BranchLevel<HB, SB, E + 1, K, BUDGET - K>::run(h, s, carry, acc, p);
+            BranchLevel<HB, SB, GQ, E + 1, K, BUDGET - K>::run(h, s, carry, acc, p);
         }
     }
 };
 
 template <int HB, int SB>
 struct BranchTile {
-    static constexpr int TH = (HB == 1) ? 8 : (HB == 2) ? 4 : (HB <= 4) ? 2 : 1;   // TH*HB <= 8 quads held
+    // k-quads whose xor words are compressed together: a 1 x 1 bit product has only 4 words per
+    // k-quad, too few for the adders to pay, so two k-quads are taken at once
+    static constexpr int GQ = (HB * SB == 1) ? 2 : 1;
+    static constexpr int TH = ((HB == 1) ? 8 : (HB == 2) ? 4 : (HB <= 4) ? 2 : 1) / GQ;   // TH*HB*GQ <= 8 quads held
     static constexpr int KQ = (SB == 1) ? 8 : (SB == 2) ? 4 : (SB <= 4) ? 2 : 1;   // k-quads per stage
     static constexpr int STAGES = 3;
     static constexpr int THREADS = 256;
     // full adders per output and k-quad: half of the 4*HB*SB xor words balances the two pipes
     // (each adder costs two logic operations and saves one population count)
-    static constexpr int CSA_BUDGET = 2 * HB * SB;
+    static constexpr int CSA_BUDGET = 2 * HB * SB * GQ;
     // the k-quads of a stage are unrolled only while the loop body stays small enough for the
     // instruction cache (about 12 instructions per plane pair per output)
     static constexpr bool UNROLL_KQ = HB * SB <= 4;
@@ -298,32 +305,38 @@ branch_kernel(const BranchParams p) {
         }
         const uint4* hs = smem + (size_t)(it % STAGES) * STAGE_QUADS;
         const uint4* ss = hs + H_QUADS;
-        auto one_quad = [&](int kq) {
-            uint4 h[TH][HB];
+        constexpr int GQ = T::GQ;
+        auto one_group = [&](int kq) {                       // k-quads kq .. kq + GQ - 1 of this stage
+            uint4 h[TH][GQ * HB];
 #pragma unroll
             for (int a = 0; a < TH; ++a)
 #pragma unroll
-                for (int i = 0; i < HB; ++i) h[a][i] = hs[(i * KQ + kq) * BH + ty + 16 * a];
+                for (int g = 0; g < GQ; ++g)
+#pragma unroll
+                    for (int i = 0; i < HB; ++i) h[a][g * HB + i] = hs[(i * KQ + kq + g) * BH + ty + 16 * a];
 #pragma unroll
             for (int b = 0; b < TS; ++b) {
-                uint4 s[SB];
+                uint4 s[GQ * SB];
 #pragma unroll
-                for (int j = 0; j < SB; ++j) s[j] = ss[(j * KQ + kq) * BS + tx + 16 * b];
+                for (int g = 0; g < GQ; ++g)
+#pragma unroll
+                    for (int j = 0; j < SB; ++j) s[g * SB + j] = ss[(j * KQ + kq + g) * BS + tx + 16 * b];
                 const uint32_t none[1] = {0u};
 #pragma unroll
                 for (int a = 0; a < TH; ++a)
-                    BranchLevel<HB, SB, 0, 0, T::CSA_BUDGET>::run(h[a], s, none, acc[a][b], p);
+                    BranchLevel<HB, SB, GQ, 0, 0, T::CSA_BUDGET>::run(h[a], s, none, acc[a][b], p);
             }
         };
-        // the last stage may hold fewer than KQ k-quads of data: skip the rest (they are all zero)
+        // the last stage may hold fewer than KQ k-quads of data: skip the rest (they are all zero;
+        // a group that is only partly live reads zero-filled quads, which add nothing)
         const int kq_live = (int)min((int64_t)KQ, kq_total - (int64_t)it * KQ);
         if (T::UNROLL_KQ) {
 #pragma unroll
-            for (int kq = 0; kq < KQ; ++kq)
-                if (kq < kq_live) one_quad(kq);
+            for (int kq = 0; kq < KQ; kq += GQ)
+                if (kq < kq_live) one_group(kq);
         } else {
 #pragma unroll 1
-            for (int kq = 0; kq < kq_live; ++kq) one_quad(kq);
+            for (int kq = 0; kq < kq_live; kq += GQ) one_group(kq);
         }
     }
     cp_async_wait<0>();
