@@ -201,6 +201,8 @@ branch_kernel(const BranchParams p) {
     __shared__ int row_ih0[MODE == kModeConv ? BS : 1];    // top-left input coordinate of the window
     __shared__ int row_iw0[MODE == kModeConv ? BS : 1];
     __shared__ int row_pix[MODE == kModeConv ? BS : 1];    // (n*H + ih0)*W + iw0: pixel index of the window origin
+    __shared__ int row_rem[MODE == kModeConv ? BS : 1];    // oh*Wo + ow: offset of the output pixel in its plane
+    __shared__ unsigned row_out[MODE == kModeConv ? BS : 1];   // bit t set: filter tap t falls outside the image
 
     const int tid = threadIdx.x;
     const int tx = tid & 15, ty = tid >> 4;
@@ -221,8 +223,16 @@ branch_kernel(const BranchParams p) {
                 row_ih0[r] = (rem / p.Wo) * p.stride - p.pad;
                 row_iw0[r] = (rem % p.Wo) * p.stride - p.pad;
                 row_pix[r] = (n * p.H + row_ih0[r]) * p.W + row_iw0[r];
+                row_rem[r] = rem;
+                unsigned outside = 0;
+                for (int t = 0; t < p.KH * p.KW; ++t) {
+                    const int ih = row_ih0[r] + t / p.KW, iw = row_iw0[r] + t % p.KW;
+                    if (ih < 0 || ih >= p.H || iw < 0 || iw >= p.W) outside |= 1u << t;
+                }
+                row_out[r] = outside;
             } else {
                 row_n[r] = -1; row_ih0[r] = -(1 << 20); row_iw0[r] = 0; row_pix[r] = 0;   // never inside the image
+                row_rem[r] = 0; row_out[r] = 0;
             }
         }
         __syncthreads();
@@ -384,17 +394,10 @@ branch_kernel(const BranchParams p) {
             const int r = tx + 16 * b;
             const int n = row_n[r];
             if (n < 0) continue;
-            const int ih0 = row_ih0[r], iw0 = row_iw0[r];
             // taps of this pixel that fall outside the image were staged as all-zero bits, i.e. as the
             // code -L_a; what they added, -L_a * tap_sum[tap][o], is taken out again so they count as 0
-            unsigned outside = 0;
-            if (p.pad > 0) {
-                for (int t = 0; t < taps; ++t) {
-                    const int ih = ih0 + t / p.KW, iw = iw0 + t % p.KW;
-                    if (ih < 0 || ih >= p.H || iw < 0 || iw >= p.W) outside |= 1u << t;
-                }
-            }
-            const int64_t rem = (s0 + r) % hw;
+            const unsigned outside = row_out[r];
+            const int64_t rem = row_rem[r];
 #pragma unroll
             for (int a = 0; a < TH; ++a) {
                 const int64_t o = h0 + ty + 16 * a;
