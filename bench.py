@@ -99,6 +99,23 @@ class ClockSampler:
         return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "reasons": sorted(reasons), "samples": len(sm)}
 
 
+def max_over_ranks(value: float, world: int, device=None) -> float:
+    """Slowest rank's figure: every rank contributes its own time, all get the maximum.
+    (The replicas share nothing else: the path has no exchange step.)"""
+    if world <= 1:
+        return float(value)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_tops(world: int, m: int, n: int, k: int, ms_per_step: float) -> float:
+    """Aggregate equivalent TOPS of `world` independent replicas that each do one m x n x k layer per step."""
+    return world * 2.0 * m * n * k / (ms_per_step * 1e-3) / 1e12
+
+
 def _workload_arrays():
     from paper_1905_13389_b200 import inputs
     c = inputs.config4(W_BITS, A_BITS, SIZE)
@@ -224,13 +241,9 @@ def run_cuda(args):
             step(True)
         t1.record()
         barrier()
-    elapsed_ms = t0.elapsed_time(t1)
-    if world > 1:
-        t = torch.tensor([elapsed_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        elapsed_ms = float(t.item())
+    elapsed_ms = max_over_ranks(t0.elapsed_time(t1), world, dev)
     ms_per_step = elapsed_ms / args.steps
-    value = world * 2.0 * m * n * k / (ms_per_step * 1e-3) / 1e12
+    value = whole_job_tops(world, m, n, k, ms_per_step)
 
     gemm_ms = statistics.mean(a.elapsed_time(b) for a, b in gemm_events)
     enc_ms = statistics.mean(a.elapsed_time(b) for a, b in enc_events)
@@ -255,12 +268,8 @@ def run_cuda(args):
         mpq.linear_host(xh, wh, A_BITS, W_BITS, out_i32_host=oi, out_f32_host=of, workspace=ws)
     t1.record()
     barrier()
-    e2e_ms = t0.elapsed_time(t1)
-    if world > 1:
-        t = torch.tensor([e2e_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
-    e2e_value = world * 2.0 * m * n * k / (e2e_ms / e2e_steps * 1e-3) / 1e12
+    e2e_ms = max_over_ranks(t0.elapsed_time(t1), world, dev)
+    e2e_value = whole_job_tops(world, m, n, k, e2e_ms / e2e_steps)
 
     if rank == 0:
         line = {
