@@ -204,6 +204,7 @@ branch_kernel(const BranchParams p) {
     __shared__ int row_rem[MODE == kModeConv ? BS : 1];    // oh*Wo + ow: offset of the output pixel in its plane
     __shared__ unsigned row_out[MODE == kModeConv ? BS : 1];   // bit t set: filter tap t falls outside the image
 
+    chain_entry();
     const int tid = threadIdx.x;
     const int tx = tid & 15, ty = tid >> 4;
     const int64_t s_tiles = ceil_div(p.streamed_rows, BS);
@@ -434,8 +435,7 @@ static int launch_branch(const BranchParams& p, cudaStream_t st) {
     }
     const int64_t blocks = ceil_div(p.streamed_rows, BS) * ceil_div(p.held_rows, BH);
     if (blocks <= 0 || blocks > 0x7fffffffLL) return MPQ_ERR_BAD_SHAPE;
-    kern<<<(unsigned)blocks, 256, smem_bytes, st>>>(p);
-    return launch_status();
+    return launch_chained(kern, (unsigned)blocks, 256, smem_bytes, st, p);
 }
 
 // Streamed-side tile width (16*TS items): the widest tile has the least shared-memory traffic per

@@ -18,6 +18,7 @@ template <int ACT, bool VEC4>
 __global__ void __launch_bounds__(kAbsmaxThreads)
 absmax_kernel(const float* __restrict__ x, int64_t k, int64_t ldx, int64_t chunks_per_row,
               int per_row, float* __restrict__ out) {
+    chain_entry();
     const int64_t row = blockIdx.x / chunks_per_row;
     const int64_t e0 = (blockIdx.x % chunks_per_row) * kAbsmaxChunk;
     const float* xr = x + row * ldx;
@@ -91,6 +92,7 @@ encode_rows_kernel(const float* __restrict__ x, int64_t rows, int64_t k, int64_t
                    uint32_t* __restrict__ planes, int64_t rw, int64_t segs_per_row,
                    int vec_ok, uint32_t two) {
     __shared__ __align__(16) float stage[kEncodeThreads / 32][32 * kStageRow];
+    chain_entry();
     const int64_t warp = (int64_t)blockIdx.x * (kEncodeThreads / 32) + (threadIdx.x >> 5);
     if (warp >= rows * segs_per_row) return;
     const int lane = threadIdx.x & 31;
@@ -187,6 +189,7 @@ __global__ void __launch_bounds__(kEncodeThreads)
 encode_nchw_kernel(const float* __restrict__ x, int N, int C, int64_t HW,
                    const float* __restrict__ scale, uint32_t* __restrict__ planes,
                    int64_t pix_blocks, int64_t total_warps, uint32_t two) {
+    chain_entry();
     const int64_t warp = (int64_t)blockIdx.x * (kEncodeThreads / 32) + (threadIdx.x >> 5);
     if (warp >= total_warps) return;
     const int lane = threadIdx.x & 31;
@@ -282,6 +285,7 @@ __global__ void tap_sums_kernel(const float* __restrict__ w, int O, int C, int t
 
 __global__ void add_relu_kernel(const float* __restrict__ a, const float* __restrict__ b,
                                 float* __restrict__ y, int64_t n) {
+    chain_entry();
     const int64_t stride = (int64_t)gridDim.x * blockDim.x;
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride) {
         const float v = b ? __fadd_rn(a[i], b[i]) : a[i];
@@ -313,9 +317,8 @@ struct EncodeRowsLauncher {
         if (blocks > 0x7fffffffLL) return MPQ_ERR_BAD_SHAPE;
         // the lane-local path copies 16-byte chunks: every row start must be 16-byte aligned
         const int vec_ok = aligned16(x) && (ldx % 4 == 0 || rows == 1);
-        encode_rows_kernel<BITS, ACT><<<(unsigned)blocks, kEncodeThreads, 0, st>>>(
-            x, rows, k, ldx, scale, per_row, planes, rw, segs, vec_ok, 2u);
-        return launch_status();
+        return launch_chained(encode_rows_kernel<BITS, ACT>, (unsigned)blocks, kEncodeThreads, 0, st,
+                              x, rows, k, ldx, scale, per_row, planes, rw, segs, vec_ok, 2u);
     }
 };
 
@@ -326,9 +329,8 @@ struct EncodeNchwLauncher {
         const int64_t warps = pix_blocks * (C / 32) * N;
         const int64_t blocks = ceil_div(warps, kEncodeThreads / 32);
         if (blocks > 0x7fffffffLL) return MPQ_ERR_BAD_SHAPE;
-        encode_nchw_kernel<BITS, ACT><<<(unsigned)blocks, kEncodeThreads, 0, st>>>(
-            x, N, C, HW, scale, planes, pix_blocks, warps, 2u);
-        return launch_status();
+        return launch_chained(encode_nchw_kernel<BITS, ACT>, (unsigned)blocks, kEncodeThreads, 0, st,
+                              x, N, C, HW, scale, planes, pix_blocks, warps, 2u);
     }
 };
 
@@ -350,11 +352,10 @@ extern "C" int mpq_absmax(const float* x, int64_t rows, int64_t k, int64_t ldx, 
     const int64_t blocks = rows * chunks;
     if (blocks > 0x7fffffffLL) return MPQ_ERR_BAD_SHAPE;
     const bool vec4 = aligned16(x) && (ldx % 4 == 0);
-#define MPQ_LAUNCH(A, V) absmax_kernel<A, V><<<(unsigned)blocks, kAbsmaxThreads, 0, st>>>(x, k, ldx, chunks, per_row, scale_out)
-    if (act == MPQ_ACT_HRELU) { if (vec4) MPQ_LAUNCH(MPQ_ACT_HRELU, true); else MPQ_LAUNCH(MPQ_ACT_HRELU, false); }
-    else                      { if (vec4) MPQ_LAUNCH(MPQ_ACT_HTANH, true); else MPQ_LAUNCH(MPQ_ACT_HTANH, false); }
+#define MPQ_LAUNCH(A, V) launch_chained(absmax_kernel<A, V>, (unsigned)blocks, kAbsmaxThreads, 0, st, x, k, ldx, chunks, per_row, scale_out)
+    if (act == MPQ_ACT_HRELU) return vec4 ? MPQ_LAUNCH(MPQ_ACT_HRELU, true) : MPQ_LAUNCH(MPQ_ACT_HRELU, false);
+    return vec4 ? MPQ_LAUNCH(MPQ_ACT_HTANH, true) : MPQ_LAUNCH(MPQ_ACT_HTANH, false);
 #undef MPQ_LAUNCH
-    return launch_status();
 }
 
 extern "C" int mpq_encode(const float* x, int64_t rows, int64_t k, int64_t ldx,
@@ -400,6 +401,5 @@ extern "C" int mpq_add_relu(const float* a, const float* b, float* y, int64_t n,
     if (!a || !y) return MPQ_ERR_NULL;
     if (n <= 0) return MPQ_ERR_BAD_SHAPE;
     const int64_t blocks = min((int64_t)148 * 16, ceil_div(n, 256));
-    add_relu_kernel<<<(unsigned)blocks, 256, 0, (cudaStream_t)stream>>>(a, b, y, n);
-    return launch_status();
+    return launch_chained(add_relu_kernel, (unsigned)blocks, 256, 0, (cudaStream_t)stream, a, b, y, n);
 }

@@ -21,6 +21,7 @@ __global__ void __launch_bounds__(kStemTile* kStemTile)
 stem_conv7x7_kernel(const float* __restrict__ x, const float* __restrict__ w, float* __restrict__ y,
                     int N, int H, int W, int Ho, int Wo, int relu) {
     extern __shared__ __align__(16) float smem[];
+    chain_entry();
     float* ws = smem;                                   // [147][64]
     float* xs = smem + kStemTaps * kStemO;              // [3][37][38]
     constexpr int kRow = kStemPatch + 1;
@@ -85,6 +86,7 @@ stem_conv7x7_kernel(const float* __restrict__ x, const float* __restrict__ w, fl
 // 3x3 max-pool, stride 2, pad 1 (padding never wins: the window always holds a real element).
 __global__ void maxpool3x3s2_kernel(const float* __restrict__ x, float* __restrict__ y,
                                     int64_t planes, int H, int W, int Ho, int Wo) {
+    chain_entry();
     const int64_t total = planes * Ho * Wo;
     const int64_t stride = (int64_t)gridDim.x * blockDim.x;
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += stride) {
@@ -125,9 +127,8 @@ extern "C" int mpq_stem_conv7x7(const float* x, const float* w, float* y, int N,
             return MPQ_ERR_CUDA;
         configured[dev] = true;
     }
-    stem_conv7x7_kernel<<<(unsigned)blocks, kStemTile * kStemTile, smem, (cudaStream_t)stream>>>(
-        x, w, y, N, H, W, Ho, Wo, relu);
-    return launch_status();
+    return launch_chained(stem_conv7x7_kernel, (unsigned)blocks, kStemTile * kStemTile, smem, (cudaStream_t)stream,
+                          x, w, y, N, H, W, Ho, Wo, relu);
 }
 
 extern "C" int mpq_maxpool3x3s2(const float* x, float* y, int N, int C, int H, int W, void* stream) {
@@ -136,6 +137,6 @@ extern "C" int mpq_maxpool3x3s2(const float* x, float* y, int N, int C, int H, i
     const int Ho = (H + 2 - 3) / 2 + 1, Wo = (W + 2 - 3) / 2 + 1;
     const int64_t total = (int64_t)N * C * Ho * Wo;
     const int64_t blocks = min((int64_t)148 * 16, ceil_div(total, 256));
-    maxpool3x3s2_kernel<<<(unsigned)blocks, 256, 0, (cudaStream_t)stream>>>(x, y, (int64_t)N * C, H, W, Ho, Wo);
-    return launch_status();
+    return launch_chained(maxpool3x3s2_kernel, (unsigned)blocks, 256, 0, (cudaStream_t)stream,
+                          x, y, (int64_t)N * C, H, W, Ho, Wo);
 }
