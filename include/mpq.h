@@ -171,8 +171,12 @@ int mpq_linear_static(const float* x, const float* w, int64_t m, int64_t n, int6
 
 /* The same layer from HOST buffers: copies x_host and w_host into the device workspace, runs
  * mpq_linear there, and copies out_i32_host / out_f32_host [m x n] back (either may be NULL, not
- * both).  Host buffers should be pinned for the copies to be asynchronous.  The call returns
- * after the stream has drained (it synchronizes `stream`).
+ * both).  Host buffers should be pinned for the copies to be asynchronous.  The weights are
+ * copied and encoded first (that work overlaps the activations' copy), and the product runs in
+ * row blocks whose results are copied back on a helper stream while the next block is computed
+ * (one helper stream and five events per device, created by the first call on that device and
+ * kept until exit; two calls on one device must not overlap).  The call returns after everything
+ * has drained (it synchronizes `stream`).
  * workspace: device memory of at least mpq_linear_host_workspace() bytes, 256-byte aligned. */
 int64_t mpq_linear_host_workspace(int64_t m, int64_t n, int64_t k, int a_bits, int w_bits);
 int mpq_linear_host(const float* x_host, const float* w_host, int64_t m, int64_t n, int64_t k,

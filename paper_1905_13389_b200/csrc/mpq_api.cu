@@ -150,6 +150,37 @@ extern "C" int64_t mpq_linear_host_workspace(int64_t m, int64_t n, int64_t k, in
     return host_layout(m, n, k, a_bits, w_bits).total;
 }
 
+// Copy-out helper of mpq_linear_host: one extra stream and a few events per device, created on
+// the first call on that device and kept until the process exits, so that finished row blocks
+// travel to the host while the next block is still being computed.
+namespace {
+constexpr int kHostBlocks = 4;
+struct HostPipe {
+    cudaStream_t copy_stream = nullptr;
+    cudaEvent_t block_done[kHostBlocks] = {};
+    cudaEvent_t copies_done = nullptr;
+    bool ready = false;
+};
+HostPipe g_host_pipe[kMaxDevices];
+std::mutex g_host_pipe_mutex;
+
+int host_pipe(HostPipe** out) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return MPQ_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(g_host_pipe_mutex);
+    HostPipe& hp = g_host_pipe[dev];
+    if (!hp.ready) {
+        if (cudaStreamCreateWithFlags(&hp.copy_stream, cudaStreamNonBlocking) != cudaSuccess) return MPQ_ERR_CUDA;
+        for (int i = 0; i < kHostBlocks; ++i)
+            if (cudaEventCreateWithFlags(&hp.block_done[i], cudaEventDisableTiming) != cudaSuccess) return MPQ_ERR_CUDA;
+        if (cudaEventCreateWithFlags(&hp.copies_done, cudaEventDisableTiming) != cudaSuccess) return MPQ_ERR_CUDA;
+        hp.ready = true;
+    }
+    *out = &hp;
+    return MPQ_OK;
+}
+}  // namespace
+
 extern "C" int mpq_linear_host(const float* x_host, const float* w_host, int64_t m, int64_t n, int64_t k,
                                int a_bits, int w_bits, int a_act, int w_mode,
                                int32_t* out_i32_host, float* out_f32_host,
@@ -166,11 +197,37 @@ extern "C" int mpq_linear_host(const float* x_host, const float* w_host, int64_t
     float* w = reinterpret_cast<float*>(ws + L.w);
     int32_t* oi = out_i32_host ? reinterpret_cast<int32_t*>(ws + L.out_i32) : nullptr;
     float* of = out_f32_host ? reinterpret_cast<float*>(ws + L.out_f32) : nullptr;
-    if (cudaMemcpyAsync(x, x_host, (size_t)m * k * 4, cudaMemcpyHostToDevice, st) != cudaSuccess) return MPQ_ERR_CUDA;
+    // weights first: their range and planes are computed while the activations are still in flight
+    const LinearScratch S = linear_scratch(m, n, k, a_bits, w_bits);
+    char* sc = ws + L.scratch;
+    float* s_a = reinterpret_cast<float*>(sc + S.s_a);
+    float* s_w = reinterpret_cast<float*>(sc + S.s_w);
+    uint32_t* ap = reinterpret_cast<uint32_t*>(sc + S.a_planes);
+    uint32_t* wp = reinterpret_cast<uint32_t*>(sc + S.w_planes);
     if (cudaMemcpyAsync(w, w_host, (size_t)n * k * 4, cudaMemcpyHostToDevice, st) != cudaSuccess) return MPQ_ERR_CUDA;
-    if ((rc = linear_on_scratch(x, w, m, n, k, a_bits, w_bits, a_act, w_mode, oi, of, ws + L.scratch, st)) != MPQ_OK) return rc;
-    if (oi && cudaMemcpyAsync(out_i32_host, oi, (size_t)m * n * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess) return MPQ_ERR_CUDA;
-    if (of && cudaMemcpyAsync(out_f32_host, of, (size_t)m * n * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess) return MPQ_ERR_CUDA;
+    if ((rc = mpq_absmax(w, n, k, k, w_mode, MPQ_ACT_HTANH, s_w, st)) != MPQ_OK) return rc;
+    if ((rc = mpq_encode(w, n, k, k, s_w, w_mode, MPQ_ACT_HTANH, w_bits, wp, st)) != MPQ_OK) return rc;
+    if (cudaMemcpyAsync(x, x_host, (size_t)m * k * 4, cudaMemcpyHostToDevice, st) != cudaSuccess) return MPQ_ERR_CUDA;
+    if ((rc = mpq_absmax(x, m, k, k, MPQ_SCALE_PER_TENSOR, a_act, s_a, st)) != MPQ_OK) return rc;
+    if ((rc = mpq_encode(x, m, k, k, s_a, MPQ_SCALE_PER_TENSOR, a_act, a_bits, ap, st)) != MPQ_OK) return rc;
+    // the product in row blocks; each finished block is copied out on the helper stream
+    HostPipe* hp = nullptr;
+    if ((rc = host_pipe(&hp)) != MPQ_OK) return rc;
+    const int blocks = m >= 1024 ? kHostBlocks : 1;
+    const int64_t per = ((m + blocks - 1) / blocks + 63) / 64 * 64;
+    for (int b = 0; b < blocks; ++b) {
+        const int64_t r0 = (int64_t)b * per;
+        if (r0 >= m) break;
+        const int64_t rows = (r0 + per <= m) ? per : m - r0;
+        if ((rc = gemm_rows(ap, a_bits, wp, w_bits, m, r0, rows, n, k, oi, of, n, s_a, s_w, w_mode, st)) != MPQ_OK) return rc;
+        if (cudaEventRecord(hp->block_done[b], st) != cudaSuccess) return MPQ_ERR_CUDA;
+        if (cudaStreamWaitEvent(hp->copy_stream, hp->block_done[b], 0) != cudaSuccess) return MPQ_ERR_CUDA;
+        const size_t off = (size_t)r0 * n, bytes = (size_t)rows * n * 4;
+        if (oi && cudaMemcpyAsync(out_i32_host + off, oi + off, bytes, cudaMemcpyDeviceToHost, hp->copy_stream) != cudaSuccess) return MPQ_ERR_CUDA;
+        if (of && cudaMemcpyAsync(out_f32_host + off, of + off, bytes, cudaMemcpyDeviceToHost, hp->copy_stream) != cudaSuccess) return MPQ_ERR_CUDA;
+    }
+    if (cudaEventRecord(hp->copies_done, hp->copy_stream) != cudaSuccess) return MPQ_ERR_CUDA;
+    if (cudaStreamWaitEvent(st, hp->copies_done, 0) != cudaSuccess) return MPQ_ERR_CUDA;
     return cudaStreamSynchronize(st) == cudaSuccess ? MPQ_OK : MPQ_ERR_CUDA;
 }
 

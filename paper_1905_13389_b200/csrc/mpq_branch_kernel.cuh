@@ -28,7 +28,8 @@ enum { kModeGemm = 0, kModeConv = 1 };
 struct BranchParams {
     const uint32_t* held;      // GEMM: A planes [HB][m][rw];      CONV: weight planes [HB][O][rw]
     const uint32_t* streamed;  // GEMM: B planes [SB][n][rw];      CONV: x planes [SB][N][H][W][Cw]
-    int64_t held_rows;         // GEMM: m;  CONV: O
+    int64_t held_rows;         // GEMM: m (rows computed by this launch);  CONV: O
+    int64_t held_plane_rows;   // rows between two planes of the held operand in memory (>= held_rows)
     int64_t streamed_rows;     // GEMM: n;  CONV: N*Ho*Wo
     int64_t rw;                // words per packed row (GEMM: both operands; CONV: weight rows)
     int64_t k;                 // elements per dot product (CONV: KH*KW*C)
@@ -250,7 +251,7 @@ branch_kernel(const BranchParams p) {
                 const int kq = id % KQ, row = (id / KQ) % BH, plane = id / (KQ * BH);
                 const int64_t grow = h0 + row, gkq = kq0 + kq;
                 const bool ok = grow < p.held_rows && gkq < kq_total;
-                const uint32_t* src = ok ? p.held + ((int64_t)plane * p.held_rows + grow) * p.rw + gkq * 4 : p.held;
+                const uint32_t* src = ok ? p.held + ((int64_t)plane * p.held_plane_rows + grow) * p.rw + gkq * 4 : p.held;
                 cp_async_16(hs + (plane * KQ + kq) * BH + row, src, ok);
             }
         }

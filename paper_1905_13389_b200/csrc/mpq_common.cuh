@@ -18,6 +18,13 @@ inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 
 
 inline int launch_status() { return cudaGetLastError() == cudaSuccess ? MPQ_OK : MPQ_ERR_CUDA; }
 
+// Rows [row0, row0 + rows) of the layer product (mpq_gemm on a row block of A): lets a caller
+// overlap the copy-out of finished rows with the product of the next ones.
+int gemm_rows(const uint32_t* a_planes, int a_bits, const uint32_t* b_planes, int b_bits,
+              int64_t m_total, int64_t row0, int64_t rows, int64_t n, int64_t k,
+              int32_t* c_i32, float* c_f32, int64_t ldc,
+              const float* a_scale, const float* b_scale, int b_mode, cudaStream_t stream);
+
 // ---- Chained launches (programmatic dependent launch) --------------------------------------
 // A layer is a chain of short kernels on one stream (range, encode, product, add).  Launched
 // with the programmatic-serialization attribute, a kernel's blocks may become resident while the

@@ -48,25 +48,36 @@ static bool int32_headroom(int64_t k, int a_bits, int w_bits) {
 
 using namespace mpq;
 
-extern "C" int mpq_gemm(const uint32_t* a_planes, int a_bits, const uint32_t* b_planes, int b_bits,
-                        int64_t m, int64_t n, int64_t k,
-                        int32_t* c_i32, float* c_f32, int64_t ldc,
-                        const float* a_scale, const float* b_scale, int b_mode, void* stream) {
+// Rows [row0, row0 + rows) of C = A * B^T, A holding m_total rows per plane.
+int mpq::gemm_rows(const uint32_t* a_planes, int a_bits, const uint32_t* b_planes, int b_bits,
+                   int64_t m_total, int64_t row0, int64_t rows, int64_t n, int64_t k,
+                   int32_t* c_i32, float* c_f32, int64_t ldc,
+                   const float* a_scale, const float* b_scale, int b_mode, cudaStream_t stream) {
     if (!a_planes || !b_planes || (!c_i32 && !c_f32)) return MPQ_ERR_NULL;
     if (c_f32 && (!a_scale || !b_scale)) return MPQ_ERR_NULL;
-    if (m <= 0 || n <= 0 || k <= 0 || ldc < n) return MPQ_ERR_BAD_SHAPE;
+    if (m_total <= 0 || n <= 0 || k <= 0 || ldc < n || row0 < 0 || rows <= 0 || row0 + rows > m_total) return MPQ_ERR_BAD_SHAPE;
     if (!bits_ok(a_bits) || !bits_ok(b_bits) ||
         (b_mode != MPQ_SCALE_PER_TENSOR && b_mode != MPQ_SCALE_PER_ROW)) return MPQ_ERR_UNSUPPORTED;
     if (!int32_headroom(k, a_bits, b_bits)) return MPQ_ERR_OVERFLOW;
     if (!aligned16(a_planes) || !aligned16(b_planes)) return MPQ_ERR_ALIGN;
     BranchParams p = {};
-    p.held = a_planes; p.streamed = b_planes;
-    p.held_rows = m; p.streamed_rows = n;
     p.rw = row_words(k); p.k = k;
-    p.out_i32 = c_i32; p.out_f32 = c_f32; p.ldc = ldc;
+    p.held = a_planes + row0 * p.rw; p.streamed = b_planes;
+    p.held_rows = rows; p.held_plane_rows = m_total; p.streamed_rows = n;
+    p.out_i32 = c_i32 ? c_i32 + row0 * ldc : nullptr;
+    p.out_f32 = c_f32 ? c_f32 + row0 * ldc : nullptr;
+    p.ldc = ldc;
     p.a_scale = a_scale; p.w_scale = b_scale; p.w_per_row = b_mode == MPQ_SCALE_PER_ROW;
     fill_pow2(p);
-    return dispatch_gemm(a_bits, b_bits, p, (cudaStream_t)stream);
+    return dispatch_gemm(a_bits, b_bits, p, stream);
+}
+
+extern "C" int mpq_gemm(const uint32_t* a_planes, int a_bits, const uint32_t* b_planes, int b_bits,
+                        int64_t m, int64_t n, int64_t k,
+                        int32_t* c_i32, float* c_f32, int64_t ldc,
+                        const float* a_scale, const float* b_scale, int b_mode, void* stream) {
+    return mpq::gemm_rows(a_planes, a_bits, b_planes, b_bits, m, 0, m, n, k, c_i32, c_f32, ldc,
+                          a_scale, b_scale, b_mode, (cudaStream_t)stream);
 }
 
 extern "C" int mpq_conv(const uint32_t* x_planes, int a_bits, int N, int C, int H, int W,
@@ -90,7 +101,7 @@ extern "C" int mpq_conv(const uint32_t* x_planes, int a_bits, int N, int C, int 
     p.held = w_planes; p.streamed = x_planes;
     p.Ho = (H + 2 * pad - KH) / stride + 1;
     p.Wo = (W + 2 * pad - KW) / stride + 1;
-    p.held_rows = O; p.streamed_rows = (int64_t)N * p.Ho * p.Wo;
+    p.held_rows = O; p.held_plane_rows = O; p.streamed_rows = (int64_t)N * p.Ho * p.Wo;
     p.rw = row_words(K); p.k = K;
     p.out_i32 = y_i32; p.out_f32 = y_f32; p.ldc = 0;
     p.a_scale = x_scale; p.w_scale = w_scale; p.w_per_row = w_mode == MPQ_SCALE_PER_ROW;

@@ -337,6 +337,24 @@ def test_linear_host(mpq, cuda):
     assert rel_close(of.numpy(), out_ref)
 
 
+def test_linear_host_row_blocks(mpq, cuda):
+    """m >= 1024: the product runs in row blocks that are copied out while the next one computes
+    (ragged last block, per-row weight ranges, both outputs, then the int32 output alone)."""
+    m, n, k = 1100, 70, 200
+    x = inputs.uniform_levels(6, 11, (m, k), 3)
+    w = inputs.uniform_levels(6, 12, (n, k), 2)
+    xh, wh = torch.from_numpy(x).pin_memory(), torch.from_numpy(w).pin_memory()
+    acc_ref, out_ref, _, _ = oracle.linear(x, w, 3, 2, w_per_row=True, a_act=oracle.HRELU)
+    oi = torch.full((m, n), -1, dtype=torch.int32).pin_memory()
+    of = torch.full((m, n), float("nan"), dtype=torch.float32).pin_memory()
+    mpq.linear_host(xh, wh, 3, 2, mpq.ACT_HRELU, mpq.SCALE_PER_ROW, out_i32_host=oi, out_f32_host=of)
+    assert np.array_equal(oi.numpy(), acc_ref)
+    assert rel_close(of.numpy(), out_ref)
+    oi.fill_(-1)
+    mpq.linear_host(xh, wh, 3, 2, mpq.ACT_HRELU, mpq.SCALE_PER_ROW, out_i32_host=oi)
+    assert np.array_equal(oi.numpy(), acc_ref)
+
+
 def test_add_relu(mpq, cuda):
     rng = np.random.default_rng(1)
     a = rng.standard_normal(10007).astype(np.float32)
