@@ -19,6 +19,7 @@
 //              fly from planes[bits][N][H][W][C/32]; consecutive tx = consecutive pixels, which
 //              is the contiguous direction of the NCHW output.
 #pragma once
+#include <type_traits>
 #include "mpq_common.cuh"
 
 namespace mpq {
@@ -46,6 +47,7 @@ struct BranchParams {
     int tap_granules;          // copies per filter tap = Cw / granule
     uint32_t tap_magic;        // ceil(2^32 / tap_granules): copy index / tap_granules by one multiply
     const int32_t* tap_sums;   // [KH*KW][O]
+    int half_tail;             // CONV: the last k-quad of a row holds data in its first two words only
     uint32_t pow2[24];         // pow2[e] = 2^e: branch weights read from the constant bank, so that
                                // "popcount * 2^e + acc" stays one integer multiply-add (FMA pipe)
 };
@@ -138,9 +140,10 @@ struct CarrySave<0, 0> {
 // Level E of one output: NC carries from the level below plus the fresh xor words of GQ k-quads;
 // BUDGET is the number of full adders still to be spent on this and the higher levels (lower
 // levels first).  h and s hold the planes of the GQ k-quads, quad-major: h[g * HB + i].
-template <int HB, int SB, int GQ, int E, int NC, int BUDGET>
+// NW = words of each k-quad that hold data (4, or 2 for the half-filled last quad of a short k).
+template <int HB, int SB, int GQ, int NW, int E, int NC, int BUDGET>
 struct BranchLevel {
-    static constexpr int NF = 4 * GQ * pairs_at_level(HB, SB, E);   // fresh xor words of this level
+    static constexpr int NF = NW * GQ * pairs_at_level(HB, SB, E);  // fresh xor words of this level
     static constexpr int N = NF + NC;
     using CS = CarrySave<N, (N >= 3 ? BUDGET : 0)>;
     static constexpr int K = CS::TOTAL;
@@ -159,13 +162,13 @@ struct BranchLevel {
                     const int j = E - i;
                     if (j >= 0 && j < SB) {
 #pragma unroll
-                        for (int c = 0; c < 4; ++c) w[n++] = quad_word(h[g * HB + i], c) ^ quad_word(s[g * SB + j], c);
+                        for (int c = 0; c < NW; ++c) w[n++] = quad_word(h[g * HB + i], c) ^ quad_word(s[g * SB + j], c);
                     }
                 }
             }
             uint32_t carry[K > 0 ? K : 1];
             CS::run(w, carry, 0, acc, p.pow2[E]);
-            BranchLevel<HB, SB, GQ, E + 1, K, BUDGET - K>::run(h, s, carry, acc, p);
+            BranchLevel<HB, SB, GQ, NW, E + 1, K, BUDGET - K>::run(h, s, carry, acc, p);
         }
     }
 };
@@ -318,7 +321,8 @@ branch_kernel(const BranchParams p) {
         const uint4* hs = smem + (size_t)(it % STAGES) * STAGE_QUADS;
         const uint4* ss = hs + H_QUADS;
         constexpr int GQ = T::GQ;
-        auto one_group = [&](int kq) {                       // k-quads kq .. kq + GQ - 1 of this stage
+        auto one_group = [&](int kq, auto words_tag) {       // k-quads kq .. kq + GQ - 1 of this stage
+            constexpr int NW = decltype(words_tag)::value;
             uint4 h[TH][GQ * HB];
 #pragma unroll
             for (int a = 0; a < TH; ++a)
@@ -336,19 +340,29 @@ branch_kernel(const BranchParams p) {
                 const uint32_t none[1] = {0u};
 #pragma unroll
                 for (int a = 0; a < TH; ++a)
-                    BranchLevel<HB, SB, GQ, 0, 0, T::CSA_BUDGET>::run(h[a], s, none, acc[a][b], p);
+                    BranchLevel<HB, SB, GQ, NW, 0, 0, (T::CSA_BUDGET * NW) / 4>::run(h[a], s, none, acc[a][b], p);
             }
         };
         // the last stage may hold fewer than KQ k-quads of data: skip the rest (they are all zero;
         // a group that is only partly live reads zero-filled quads, which add nothing)
         const int kq_live = (int)min((int64_t)KQ, kq_total - (int64_t)it * KQ);
+        // (conv only) a short k whose last k-quad is half empty: that quad is computed on two words
+        const bool half_tail = MODE == kModeConv && GQ == 1 && p.half_tail && it == n_iters - 1;
+        using Full = std::integral_constant<int, 4>;
+        using Half = std::integral_constant<int, (MODE == kModeConv && GQ == 1) ? 2 : 4>;
         if (T::UNROLL_KQ) {
 #pragma unroll
-            for (int kq = 0; kq < KQ; kq += GQ)
-                if (kq < kq_live) one_group(kq);
+            for (int kq = 0; kq < KQ; kq += GQ) {
+                if (kq < kq_live) {
+                    if (half_tail && kq == kq_live - 1) one_group(kq, Half());
+                    else one_group(kq, Full());
+                }
+            }
         } else {
+            const int full_quads = half_tail ? kq_live - 1 : kq_live;
 #pragma unroll 1
-            for (int kq = 0; kq < kq_live; kq += GQ) one_group(kq);
+            for (int kq = 0; kq < full_quads; kq += GQ) one_group(kq, Full());
+            if (half_tail) one_group(kq_live - 1, Half());
         }
     }
     cp_async_wait<0>();

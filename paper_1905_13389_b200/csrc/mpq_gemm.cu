@@ -114,6 +114,7 @@ extern "C" int mpq_conv(const uint32_t* x_planes, int a_bits, int N, int C, int 
     if ((int64_t)N * H * W >= ((int64_t)1 << 31) || (p.rw << p.granule_shift) >= 65536) return MPQ_ERR_UNSUPPORTED;
     p.tap_sums = tap_sums;
     fill_pow2(p);
+    p.half_tail = (ceil_div(K, 32) % 4 == 1 || ceil_div(K, 32) % 4 == 2) ? 1 : 0;
     // held = weights (w_bits planes), streamed = activations (a_bits planes)
     return dispatch_conv(w_bits, a_bits, p, (cudaStream_t)stream);
 }
