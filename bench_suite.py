@@ -179,7 +179,8 @@ def run_suite(dev: torch.device, hbm_gbs: float, path: str):
             Cc, Hh, Ww = net.in_shape[name]
             Ho, Wo = cv.out_hw(Hh, Ww)
             popcs = 16.0 * batch * Ho * Wo * cv.O * (cv.KH * cv.KW * Cc // 32)
-            rec.update({"span": "range + encode + conv" if "downsample" not in name else "conv",
+            rec.update({"span": "encode + conv (range, residual add and max(.,0) ride in the producers' stores)"
+                        if "downsample" not in name else "conv",
                         "frac_of_branch_peak": popcs / (t * 1e-3) / branch_peak,
                         "frac_of_plain_popc_peak": popcs / (t * 1e-3) / popc_peak})
             quant_ms += t

@@ -119,6 +119,23 @@ int mpq_conv(const uint32_t* x_planes, int a_bits, int N, int C, int H, int W,
              int32_t* y_i32, float* y_f32,
              const float* x_scale, const float* w_scale, int w_mode, void* stream);
 
+/* mpq_conv with the glue of a chained network folded into the store (the arithmetic of the layer
+ * itself is unchanged): f = float(acc) * alpha[o]; if `residual` (fp32, layout of y) f = f + residual
+ * (one rounded add); if `relu` f = max(f, 0); y_f32 = f.  If `out_max` is given, the single float it
+ * points to is raised to the largest stored max(f, 0) by an exact atomic maximum: it is the range
+ * the next layer's HReLU encoder needs (Table 1), taken while the outputs are still in registers.
+ * The caller zeroes *out_max beforehand (mpq_zero); the call never lowers it.  residual, relu and
+ * out_max need y_f32.  y_i32, when given, still receives the raw accumulators. */
+int mpq_conv_fused(const uint32_t* x_planes, int a_bits, int N, int C, int H, int W,
+                   const uint32_t* w_planes, int w_bits, const int32_t* tap_sums,
+                   int O, int KH, int KW, int stride, int pad,
+                   int32_t* y_i32, float* y_f32,
+                   const float* x_scale, const float* w_scale, int w_mode,
+                   const float* residual, int relu, float* out_max, void* stream);
+
+/* Sets `bytes` bytes of device memory to zero on the stream (ranges that kernels raise by atomic maximum). */
+int mpq_zero(void* p, int64_t bytes, void* stream);
+
 /* ---- Glue for chained layers (not part of the paper's method): y = max(a + b, 0) elementwise,
  * b may be NULL (plain ReLU).  n elements, fp32, one rounded add. */
 int mpq_add_relu(const float* a, const float* b, float* y, int64_t n, void* stream);
@@ -127,10 +144,11 @@ int mpq_add_relu(const float* a, const float* b, float* y, int64_t n, void* stre
  * layer of the network stays fp32).  Stem: x [N][3][H][W], w [64][3][7][7] -> y [N][64][Ho][Wo],
  * 7x7, stride 2, zero pad 3, Ho = (H - 1)/2 + 1; relu != 0 applies max(.,0) in the store.  Each
  * output is one chain of fused multiply-adds over (c, kh, kw) in that order.
- * Max-pool: 3x3, stride 2, pad 1: x [N][C][H][W] -> y [N][C][(H - 1)/2 + 1][(W - 1)/2 + 1]. */
+ * Max-pool: 3x3, stride 2, pad 1: x [N][C][H][W] -> y [N][C][(H - 1)/2 + 1][(W - 1)/2 + 1]; out_max
+ * (optional, zeroed by the caller) is raised to the largest max(y, 0), as in mpq_conv_fused. */
 int mpq_stem_conv7x7(const float* x, const float* w, float* y, int N, int H, int W, int relu,
                      void* stream);
-int mpq_maxpool3x3s2(const float* x, float* y, int N, int C, int H, int W, void* stream);
+int mpq_maxpool3x3s2(const float* x, float* y, int N, int C, int H, int W, float* out_max, void* stream);
 
 /* ---- Whole encoded fully-connected layer (Fig. 1 end to end: Encoder of both operands,
  * the a_bits x w_bits branches, Decoder): out = decode(encode(x) . encode(w)^T).

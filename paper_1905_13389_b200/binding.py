@@ -53,7 +53,10 @@ def lib() -> ctypes.CDLL:
         L.mpq_conv.argtypes = [P, i32, i32, i32, i32, i32, P, i32, P, i32, i32, i32, i32, i32, P, P, P, P, i32, P]
         L.mpq_add_relu.argtypes = [P, P, P, i64, P]
         L.mpq_stem_conv7x7.argtypes = [P, P, P, i32, i32, i32, i32, P]
-        L.mpq_maxpool3x3s2.argtypes = [P, P, i32, i32, i32, i32, P]
+        L.mpq_maxpool3x3s2.argtypes = [P, P, i32, i32, i32, i32, P, P]
+        L.mpq_conv_fused.argtypes = [P, i32, i32, i32, i32, i32, P, i32, P, i32, i32, i32, i32, i32, P, P, P, P, i32,
+                                     P, i32, P, P]
+        L.mpq_zero.argtypes = [P, i64, P]
         L.mpq_linear_workspace.argtypes = [i64, i64, i64, i32, i32]
         L.mpq_linear_workspace.restype = i64
         L.mpq_linear.argtypes = [P, P, i64, i64, i64, i32, i32, i32, i32, P, P, P, i64, P]
@@ -67,7 +70,7 @@ def lib() -> ctypes.CDLL:
                                            ctypes.POINTER(ctypes.c_int), P]
         L.mpq_measure_mix_peak.restype = i32
         for name in ("mpq_absmax", "mpq_encode", "mpq_encode_nchw", "mpq_encode_oihw", "mpq_gemm", "mpq_conv",
-                     "mpq_add_relu", "mpq_stem_conv7x7", "mpq_maxpool3x3s2", "mpq_linear", "mpq_linear_static", "mpq_linear_host", "mpq_measure_popc_peak"):
+                     "mpq_add_relu", "mpq_stem_conv7x7", "mpq_maxpool3x3s2", "mpq_conv_fused", "mpq_zero", "mpq_linear", "mpq_linear_static", "mpq_linear_host", "mpq_measure_popc_peak"):
             getattr(L, name).restype = i32
         _lib = L
     return _lib
@@ -179,6 +182,29 @@ def conv(x_planes: torch.Tensor, a_bits: int, N: int, C: int, H: int, W: int,
     return y_i32, y_f32
 
 
+def conv_fused(x_planes: torch.Tensor, a_bits: int, N: int, C: int, H: int, W: int,
+               w_planes: torch.Tensor, w_bits: int, tap_sums: Optional[torch.Tensor],
+               O: int, KH: int, KW: int, stride: int, pad: int,
+               y_i32: Optional[torch.Tensor], y_f32: torch.Tensor,
+               x_scale: torch.Tensor, w_scale: torch.Tensor, w_mode: int = SCALE_PER_ROW,
+               residual: Optional[torch.Tensor] = None, relu: bool = False,
+               out_max: Optional[torch.Tensor] = None):
+    """:func:`conv` with residual add, max(., 0) and the next layer's range folded into the store."""
+    _check(lib().mpq_conv_fused(_ptr(x_planes, torch.int32), a_bits, N, C, H, W, _ptr(w_planes, torch.int32), w_bits,
+                                _ptr(tap_sums, torch.int32), O, KH, KW, stride, pad,
+                                _ptr(y_i32, torch.int32), _ptr(y_f32, torch.float32),
+                                _ptr(x_scale, torch.float32), _ptr(w_scale, torch.float32), w_mode,
+                                _ptr(residual, torch.float32), int(relu), _ptr(out_max, torch.float32), _stream()),
+           "mpq_conv_fused")
+    return y_i32, y_f32
+
+
+def zero(t: torch.Tensor) -> torch.Tensor:
+    """Zeroes a device tensor on the current stream (cudaMemsetAsync)."""
+    _check(lib().mpq_zero(t.data_ptr(), t.numel() * t.element_size(), _stream()), "mpq_zero")
+    return t
+
+
 def add_relu(a: torch.Tensor, b: Optional[torch.Tensor], y: torch.Tensor) -> torch.Tensor:
     _check(lib().mpq_add_relu(_ptr(a, torch.float32), _ptr(b, torch.float32), _ptr(y, torch.float32),
                               a.numel(), _stream()), "mpq_add_relu")
@@ -198,12 +224,14 @@ def stem_conv7x7(x: torch.Tensor, w: torch.Tensor, relu: bool = True,
     return out
 
 
-def maxpool3x3s2(x: torch.Tensor, out: Optional[torch.Tensor] = None) -> torch.Tensor:
-    """3x3 max-pool, stride 2, pad 1 on [N][C][H][W]."""
+def maxpool3x3s2(x: torch.Tensor, out: Optional[torch.Tensor] = None,
+                 out_max: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """3x3 max-pool, stride 2, pad 1 on [N][C][H][W]; out_max (zeroed 1-float tensor) is raised to max(y, 0)."""
     N, C, H, W = x.shape
     if out is None:
         out = torch.empty((N, C, (H - 1) // 2 + 1, (W - 1) // 2 + 1), dtype=torch.float32, device=x.device)
-    _check(lib().mpq_maxpool3x3s2(_ptr(x, torch.float32), _ptr(out, torch.float32), N, C, H, W, _stream()),
+    _check(lib().mpq_maxpool3x3s2(_ptr(x, torch.float32), _ptr(out, torch.float32), N, C, H, W,
+                                  _ptr(out_max, torch.float32), _stream()),
            "mpq_maxpool3x3s2")
     return out
 

@@ -47,6 +47,9 @@ struct BranchParams {
     int tap_granules;          // copies per filter tap = Cw / granule
     uint32_t tap_magic;        // ceil(2^32 / tap_granules): copy index / tap_granules by one multiply
     const int32_t* tap_sums;   // [KH*KW][O]
+    const float* residual;     // CONV, optional: added to the scaled output (same layout), one rounded add
+    int relu;                  // CONV: store max(value, 0)
+    float* out_max;            // CONV, optional: raised (never lowered) to the largest stored max(value, 0)
     int half_tail;             // CONV: the last k-quad of a row holds data in its first two words only
     uint32_t pow2[24];         // pow2[e] = 2^e: branch weights read from the constant bank, so that
                                // "popcount * 2^e + acc" stays one integer multiply-add (FMA pipe)
@@ -405,6 +408,7 @@ branch_kernel(const BranchParams p) {
             if (want_f32 && o < p.held_rows)
                 alpha[a] = __fmul_rn(fa, __fdiv_rn(__ldg(p.w_scale + (p.w_per_row ? o : 0)), Lw));
         }
+        float seen_max = 0.0f;
 #pragma unroll
         for (int b = 0; b < TS; ++b) {
             const int r = tx + 16 * b;
@@ -427,8 +431,21 @@ branch_kernel(const BranchParams p) {
                 }
                 const int64_t idx = ((int64_t)n * p.O + o) * hw + rem;
                 if (p.out_i32) p.out_i32[idx] = v;
-                if (want_f32) p.out_f32[idx] = __fmul_rn((float)v, alpha[a]);
+                if (want_f32) {
+                    float f = __fmul_rn((float)v, alpha[a]);
+                    if (p.residual) f = __fadd_rn(f, __ldg(p.residual + idx));
+                    if (p.relu) f = fmaxf(f, 0.0f);
+                    p.out_f32[idx] = f;
+                    seen_max = fmaxf(seen_max, f);
+                }
             }
+        }
+        if (p.out_max) {
+            // range of the next layer's encoder, taken while the outputs are still in registers:
+            // non-negative floats order like their bit patterns, so an integer atomicMax is exact
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) seen_max = fmaxf(seen_max, __shfl_xor_sync(0xffffffffu, seen_max, off));
+            if ((tid & 31) == 0 && seen_max > 0.0f) atomicMax(reinterpret_cast<int*>(p.out_max), __float_as_int(seen_max));
         }
     }
 }

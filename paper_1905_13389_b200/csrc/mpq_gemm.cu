@@ -85,6 +85,18 @@ extern "C" int mpq_conv(const uint32_t* x_planes, int a_bits, int N, int C, int 
                         int O, int KH, int KW, int stride, int pad,
                         int32_t* y_i32, float* y_f32,
                         const float* x_scale, const float* w_scale, int w_mode, void* stream) {
+    return mpq_conv_fused(x_planes, a_bits, N, C, H, W, w_planes, w_bits, tap_sums, O, KH, KW, stride, pad,
+                          y_i32, y_f32, x_scale, w_scale, w_mode, nullptr, 0, nullptr, stream);
+}
+
+extern "C" int mpq_conv_fused(const uint32_t* x_planes, int a_bits, int N, int C, int H, int W,
+                        const uint32_t* w_planes, int w_bits, const int32_t* tap_sums,
+                        int O, int KH, int KW, int stride, int pad,
+                        int32_t* y_i32, float* y_f32,
+                        const float* x_scale, const float* w_scale, int w_mode,
+                        const float* residual, int relu, float* out_max, void* stream) {
+    if ((residual || relu || out_max) && !y_f32) return MPQ_ERR_NULL;
+
     if (!x_planes || !w_planes || (!y_i32 && !y_f32)) return MPQ_ERR_NULL;
     if (y_f32 && (!x_scale || !w_scale)) return MPQ_ERR_NULL;
     if (N <= 0 || C <= 0 || H <= 0 || W <= 0 || O <= 0) return MPQ_ERR_BAD_SHAPE;
@@ -113,6 +125,7 @@ extern "C" int mpq_conv(const uint32_t* x_planes, int a_bits, int N, int C, int 
     // the gather indexes pixels with 32-bit integers and divides copy indices below 2^16 exactly
     if ((int64_t)N * H * W >= ((int64_t)1 << 31) || (p.rw << p.granule_shift) >= 65536) return MPQ_ERR_UNSUPPORTED;
     p.tap_sums = tap_sums;
+    p.residual = residual; p.relu = relu != 0; p.out_max = out_max;
     fill_pow2(p);
     p.half_tail = (ceil_div(K, 32) % 4 == 1 || ceil_div(K, 32) % 4 == 2) ? 1 : 0;
     // held = weights (w_bits planes), streamed = activations (a_bits planes)

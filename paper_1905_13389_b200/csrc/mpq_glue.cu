@@ -85,8 +85,9 @@ stem_conv7x7_kernel(const float* __restrict__ x, const float* __restrict__ w, fl
 
 // 3x3 max-pool, stride 2, pad 1 (padding never wins: the window always holds a real element).
 __global__ void maxpool3x3s2_kernel(const float* __restrict__ x, float* __restrict__ y,
-                                    int64_t planes, int H, int W, int Ho, int Wo) {
+                                    int64_t planes, int H, int W, int Ho, int Wo, float* out_max) {
     chain_entry();
+    float seen_max = 0.0f;
     const int64_t total = planes * Ho * Wo;
     const int64_t stride = (int64_t)gridDim.x * blockDim.x;
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += stride) {
@@ -104,6 +105,12 @@ __global__ void maxpool3x3s2_kernel(const float* __restrict__ x, float* __restri
             }
         }
         y[i] = m;
+        seen_max = fmaxf(seen_max, m);
+    }
+    if (out_max) {
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) seen_max = fmaxf(seen_max, __shfl_xor_sync(0xffffffffu, seen_max, off));
+        if ((threadIdx.x & 31) == 0 && seen_max > 0.0f) atomicMax(reinterpret_cast<int*>(out_max), __float_as_int(seen_max));
     }
 }
 
@@ -131,12 +138,19 @@ extern "C" int mpq_stem_conv7x7(const float* x, const float* w, float* y, int N,
                           x, w, y, N, H, W, Ho, Wo, relu);
 }
 
-extern "C" int mpq_maxpool3x3s2(const float* x, float* y, int N, int C, int H, int W, void* stream) {
+extern "C" int mpq_maxpool3x3s2(const float* x, float* y, int N, int C, int H, int W, float* out_max,
+                                void* stream) {
     if (!x || !y) return MPQ_ERR_NULL;
     if (N <= 0 || C <= 0 || H <= 0 || W <= 0) return MPQ_ERR_BAD_SHAPE;
     const int Ho = (H + 2 - 3) / 2 + 1, Wo = (W + 2 - 3) / 2 + 1;
     const int64_t total = (int64_t)N * C * Ho * Wo;
     const int64_t blocks = min((int64_t)148 * 16, ceil_div(total, 256));
     return launch_chained(maxpool3x3s2_kernel, (unsigned)blocks, 256, 0, (cudaStream_t)stream,
-                          x, y, (int64_t)N * C, H, W, Ho, Wo);
+                          x, y, (int64_t)N * C, H, W, Ho, Wo, out_max);
+}
+
+extern "C" int mpq_zero(void* p, int64_t bytes, void* stream) {
+    if (!p) return MPQ_ERR_NULL;
+    if (bytes <= 0) return MPQ_ERR_BAD_SHAPE;
+    return cudaMemsetAsync(p, 0, (size_t)bytes, (cudaStream_t)stream) == cudaSuccess ? MPQ_OK : MPQ_ERR_CUDA;
 }

@@ -13,6 +13,12 @@ where the inner max(.,0) is the HReLU range limiter of conv2's encoder (Table 1)
 one is a single fp32 add + max.  Weights are encoded once, at construction, with one range per
 output channel.  All buffers are allocated at construction; ``forward`` only launches kernels
 on the current stream and never synchronises.
+
+With ``fused=True`` (the default) the glue rides in the convolutions' stores: conv2 adds the
+shortcut and applies max(.,0) itself, and every producer (max-pool, conv1, conv2) raises the
+range of the encoder that consumes it, so a block is  encode, conv, encode, conv (+ shortcut
+conv)  with no separate range or add kernels.  ``fused=False`` runs range, encode, conv and
+add as separate kernels; both give bit-identical results.
 """
 from __future__ import annotations
 
@@ -50,10 +56,11 @@ class _QConv:
 class QuantResNet18Stack:
     def __init__(self, weights: Dict[str, np.ndarray], batch: int, size: int = 224,
                  a_bits: int = 4, w_bits: int = 4, device: Optional[torch.device] = None,
-                 keep_int32: bool = False):
+                 keep_int32: bool = False, fused: bool = True):
         dev = device or torch.device("cuda", torch.cuda.current_device())
         self.dev, self.batch, self.size, self.a_bits, self.w_bits = dev, batch, size, a_bits, w_bits
         self.keep_int32 = keep_int32
+        self.fused = fused
         up = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(dev)
         self.stem_w = up(weights["conv1"])
         self.convs: Dict[str, _QConv] = {}
@@ -69,6 +76,7 @@ class QuantResNet18Stack:
         self.stem_out = f32(batch, 64, h1, h1)
         self.pooled = f32(batch, 64, h2, h2)
         # per-convolution buffers: range, packed input planes, fp32 output (and int32 when asked)
+        self.scales = f32(2 * len(BLOCKS))          # one range per encoder, contiguous: zeroed once per forward
         self.x_scale: Dict[str, torch.Tensor] = {}
         self.x_planes: Dict[str, torch.Tensor] = {}
         self.y: Dict[str, torch.Tensor] = {}
@@ -80,7 +88,7 @@ class QuantResNet18Stack:
             c1, c2 = self.convs[blk + ".conv1"], self.convs[blk + ".conv2"]
             Ho, _ = c1.out_hw(H, H)
             for name, C, Hin, conv in ((blk + ".conv1", cin, H, c1), (blk + ".conv2", cout, Ho, c2)):
-                self.x_scale[name] = f32(1)
+                self.x_scale[name] = self.scales[len(self.x_scale):len(self.x_scale) + 1]
                 self.x_planes[name] = torch.empty((a_bits, batch, Hin, Hin, C // 32), dtype=torch.int32, device=dev)
                 oh, _ = conv.out_hw(Hin, Hin)
                 self.y[name] = f32(batch, conv.O, oh, oh)
@@ -116,7 +124,7 @@ class QuantResNet18Stack:
     def forward(self, x: torch.Tensor, events: Optional[dict] = None) -> torch.Tensor:
         """x [batch][3][size][size] fp32 on the device -> output of the last block, fp32.
         With ``events`` (a dict), CUDA events are recorded around every layer:
-        events[name] = (start, end); an encoded layer's span covers its range + encode + conv
+        events[name] = (start, end); an encoded layer's span covers its (range +) encode + conv
         (the shortcut convolution reuses conv1's packed input, so its span is the conv alone)."""
         def span(name, fn):
             if events is None:
@@ -128,6 +136,8 @@ class QuantResNet18Stack:
             events[name] = (e0, e1)
             return r
 
+        if self.fused:
+            return self._forward_fused(x, span)
         span("stem", lambda: mpq.stem_conv7x7(x, self.stem_w, True, out=self.stem_out))
         cur = span("maxpool", lambda: mpq.maxpool3x3s2(self.stem_out, out=self.pooled))
         for blk, cin, cout, stride, has_ds in BLOCKS:
@@ -145,4 +155,35 @@ class QuantResNet18Stack:
             u = span(n2, second)
             shortcut = span(nd, lambda: self._conv(nd, enc["p"], enc["s"])) if has_ds else cur
             cur = span(blk + ".add_relu", lambda: mpq.add_relu(u, shortcut, self.block_out[blk]))
+        return cur
+
+    def _conv_fused(self, name, planes, scale, out, residual, relu, out_max):
+        c = self.convs[name]
+        C, H, W = self.in_shape[name]
+        mpq.conv_fused(planes, self.a_bits, self.batch, C, H, W, c.w_planes, self.w_bits, c.tap_sums,
+                       c.O, c.KH, c.KW, c.stride, c.pad, self.y_i32.get(name), out,
+                       scale, c.w_scale, mpq.SCALE_PER_ROW, residual, relu, out_max)
+        return out
+
+    def _forward_fused(self, x, span):
+        mpq.zero(self.scales)
+        span("stem", lambda: mpq.stem_conv7x7(x, self.stem_w, True, out=self.stem_out))
+        first_scale = self.x_scale[BLOCKS[0][0] + ".conv1"]
+        cur = span("maxpool", lambda: mpq.maxpool3x3s2(self.stem_out, out=self.pooled, out_max=first_scale))
+        for bi, (blk, cin, cout, stride, has_ds) in enumerate(BLOCKS):
+            n1, n2, nd = blk + ".conv1", blk + ".conv2", blk + ".downsample"
+            s1, s2 = self.x_scale[n1], self.x_scale[n2]
+            next_scale = self.x_scale[BLOCKS[bi + 1][0] + ".conv1"] if bi + 1 < len(BLOCKS) else None
+            enc = {}
+
+            def first():
+                enc["p"] = mpq.encode_nchw(cur, s1, self.a_bits, mpq.ACT_HRELU, out=self.x_planes[n1])
+                return self._conv_fused(n1, enc["p"], s1, self.y[n1], None, False, s2)
+            t = span(n1, first)
+            shortcut = span(nd, lambda: self._conv_fused(nd, enc["p"], s1, self.y[nd], None, False, None)) if has_ds else cur
+
+            def second():
+                p = mpq.encode_nchw(t, s2, self.a_bits, mpq.ACT_HRELU, out=self.x_planes[n2])
+                return self._conv_fused(n2, p, s2, self.block_out[blk], shortcut, True, next_scale)
+            cur = span(n2, second)
         return cur

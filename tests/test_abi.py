@@ -84,6 +84,13 @@ def test_host_side_argument_checks(mpq):
     assert conv(a_bits=8, w_bits=8, C=4096) == ERR_OVER    # 9 * 4096 * 255 * 255 >= 2^31
     assert L.mpq_encode_nchw(aligned, 1, 48, 4, 4, aligned, 0, 2, aligned, NULL) == ERR_UNSUP
     assert L.mpq_encode_oihw(aligned, 4, 64, 3, 3, aligned, 0, 2, aligned, NULL, NULL) == ERR_NULL
+    # fused-store convolution: the glue needs the fp32 output
+    assert L.mpq_conv_fused(aligned, 2, 1, 64, 8, 8, aligned, 2, aligned, 16, 3, 3, 1, 1, aligned, NULL,
+                            NULL, NULL, 0, aligned, 1, NULL, NULL) == ERR_NULL
+    assert L.mpq_zero(NULL, 4, NULL) == ERR_NULL and L.mpq_zero(aligned, 0, NULL) == ERR_SHAPE
+    assert L.mpq_stem_conv7x7(NULL, aligned, aligned, 1, 8, 8, 1, NULL) == ERR_NULL
+    assert L.mpq_maxpool3x3s2(aligned, aligned, 0, 4, 8, 8, NULL, NULL) == ERR_SHAPE
+    assert L.mpq_measure_mix_peak(9, None, None, None, NULL) == ERR_UNSUP
     # whole-layer calls
     assert mpq.linear_workspace(4, 0, 4, 2, 2) == 0
     lw = mpq.linear_workspace(64, 64, 512, 2, 2)

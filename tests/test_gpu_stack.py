@@ -48,12 +48,15 @@ def _oracle_block(x, ws, blk, stride, has_ds, a_bits, w_bits):
     return res, np.maximum(u + sc, np.float32(0))
 
 
+@pytest.mark.parametrize("fused", [False, True])
 @pytest.mark.parametrize("a_bits,w_bits", [(4, 4), (2, 3)])
-def test_stack_small_chain_elementwise(mpq, cuda, a_bits, w_bits):
+def test_stack_small_chain_elementwise(mpq, cuda, a_bits, w_bits, fused):
+    """fused=False: range, encode, conv, add as separate kernels; fused=True: residual add, max(.,0)
+    and the next encoder's range folded into the convolutions' stores.  Same results either way."""
     batch, size = 2, 64
     ws = inputs.config5_weights()
     x = inputs.config5_input(batch, size)
-    net = QuantResNet18Stack(ws, batch, size, a_bits, w_bits, cuda, keep_int32=True)
+    net = QuantResNet18Stack(ws, batch, size, a_bits, w_bits, cuda, keep_int32=True, fused=fused)
     out = net.forward(torch.from_numpy(x).to(cuda))
     torch.cuda.synchronize()
     cur = net.pooled.cpu().numpy()                         # the oracle chain starts from the stem's output
@@ -62,7 +65,8 @@ def test_stack_small_chain_elementwise(mpq, cuda, a_bits, w_bits):
         res, cur = _oracle_block(cur, ws, blk, stride, has_ds, a_bits, w_bits)
         for name, (acc, ref) in res.items():
             assert np.array_equal(net.y_i32[name].cpu().numpy(), acc), name
-            assert rel_close(net.y[name].cpu().numpy(), ref), name
+            if not (fused and name.endswith("conv2")):      # fused: conv2 stores the block output only
+                assert rel_close(net.y[name].cpu().numpy(), ref), name
         assert np.array_equal(net.block_out[blk].cpu().numpy(), cur), blk
         assert np.unique(res[blk + ".conv2"][0]).size > 16
     assert np.array_equal(out.cpu().numpy(), cur)
@@ -73,7 +77,7 @@ def test_stack_full_size_sampled(mpq, cuda):
     timed, on 40 sampled outputs (image corners and borders included) computed one by one."""
     batch, size, a_bits, w_bits = 128, 224, 4, 4
     ws = inputs.config5_weights()
-    net = QuantResNet18Stack(ws, batch, size, a_bits, w_bits, cuda, keep_int32=True)
+    net = QuantResNet18Stack(ws, batch, size, a_bits, w_bits, cuda, keep_int32=True, fused=True)
     net.forward(torch.from_numpy(inputs.config5_input(batch, size)).to(cuda))
     torch.cuda.synchronize()
     rng = np.random.default_rng(5)
@@ -82,6 +86,7 @@ def test_stack_full_size_sampled(mpq, cuda):
         jobs = [(blk + ".conv1", layer_in), (blk + ".conv2", net.y[blk + ".conv1"])]
         if has_ds:
             jobs.append((blk + ".downsample", layer_in))
+        shortcut = (net.y[blk + ".downsample"] if has_ds else layer_in).cpu().numpy()
         for name, xin in jobs:
             conv = net.convs[name]
             x = xin.cpu().numpy()
@@ -91,7 +96,8 @@ def test_stack_full_size_sampled(mpq, cuda):
             qx = oracle.quantize(x, s_a, a_bits, act=oracle.HRELU)
             qw = oracle.quantize(ws[name], s_w, w_bits, per_row=True)
             yi = net.y_i32[name].cpu().numpy()
-            yf = net.y[name].cpu().numpy()
+            is_conv2 = name.endswith("conv2")            # fused: stored as max(conv + shortcut, 0) in the block output
+            yf = (net.block_out[blk] if is_conv2 else net.y[name]).cpu().numpy()
             _, O, Ho, Wo = yi.shape
             pts = [(0, 0, 0, 0), (batch - 1, O - 1, Ho - 1, Wo - 1), (1, 1, 0, Wo - 1), (2, O // 2, Ho - 1, 0)]
             pts += [tuple(int(v) for v in (rng.integers(batch), rng.integers(O), rng.integers(Ho), rng.integers(Wo)))
@@ -100,5 +106,7 @@ def test_stack_full_size_sampled(mpq, cuda):
                 acc = oracle.conv_at(qx, qw, conv.stride, conv.pad, b, o, oh, ow)
                 assert int(yi[b, o, oh, ow]) == acc, (name, b, o, oh, ow)
                 ref = oracle.scale(np.array([[acc]], np.int32), s_a[0], s_w[o:o + 1], a_bits, w_bits)[0, 0]
+                if is_conv2:
+                    ref = max(np.float32(ref) + shortcut[b, o, oh, ow], np.float32(0))
                 assert abs(float(yf[b, o, oh, ow]) - float(ref)) <= 1e-5 * abs(float(ref)), (name, b, o, oh, ow)
         layer_in = net.block_out[blk]
