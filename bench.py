@@ -116,6 +116,13 @@ def whole_job_tops(world: int, m: int, n: int, k: int, ms_per_step: float) -> fl
     return world * 2.0 * m * n * k / (ms_per_step * 1e-3) / 1e12
 
 
+def _config():
+    """The workload both arms report on (the reference arm times a bounded sample of it)."""
+    return {"workload": "gemm_w2a2_4096", "m": SIZE, "n": SIZE, "k": SIZE, "a_bits": A_BITS, "w_bits": W_BITS,
+            "step": "absmax x2 + encode x2 + branch-fused GEMM (int32 + scaled fp32 out)",
+            "l2": "fp32 inputs (128 MiB) and outputs (128 MiB) per step exceed the 126 MB L2; no flush"}
+
+
 def _workload_arrays():
     from paper_1905_13389_b200 import inputs
     c = inputs.config4(W_BITS, A_BITS, SIZE)
@@ -162,8 +169,7 @@ def run_reference(args):
         "impl": "reference", "metric": METRIC, "value": tops, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": min(args.warmup, 1), "ms_per_step": dt * 1e3, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "int32", "data": "synthetic",
-        "config": {"workload": "gemm_w2a2_4096 (bounded sample: %d rows per step)" % rows, "m": SIZE, "n": SIZE, "k": SIZE,
-                   "a_bits": A_BITS, "w_bits": W_BITS},
+        "config": _config(),
         "cpu_baseline": {"value": tops, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": tops, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -295,10 +301,7 @@ def run_cuda(args):
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "int32", "data": "synthetic",
-            "config": {"workload": "gemm_w2a2_4096", "m": m, "n": n, "k": k, "a_bits": A_BITS, "w_bits": W_BITS,
-                       "step": "absmax x2 + encode x2 + branch-fused GEMM (int32 + scaled fp32 out)",
-                       "l2": "fp32 inputs (128 MiB) and outputs (128 MiB) per step exceed the 126 MB L2; no flush",
-                       "binary_tops": value * A_BITS * W_BITS},
+            "config": dict(_config(), binary_tops=value * A_BITS * W_BITS),
             "roofline": {"bound": "alu", "kernel": "branch_kernel<2,2,8,gemm> (XOR + carry-save + POPC GEMM)",
                          "achieved": achieved / 1e9, "peak": branch_peak / 1e9, "unit": "Gpopc/s",
                          "frac": achieved / branch_peak, "traffic": GEMM_DRAM_TRAFFIC_BYTES,
