@@ -294,6 +294,44 @@ def test_conv_config3(mpq, cuda):
     _conv_case(mpq, cuda, c["x"], c["w"], 3, 3, 1, 1)
 
 
+@pytest.mark.parametrize("C,ksz,stride,pad", [(64, 3, 1, 1), (128, 1, 2, 0), (32, 3, 2, 1)])
+def test_conv_fused_store(mpq, cuda, C, ksz, stride, pad):
+    """Residual add, max(.,0) and the running range folded into the store: same numbers as the
+    separate steps (oracle convolution, one fp32 add, max), and the range equals their maximum."""
+    rng = np.random.default_rng(C + ksz)
+    x = inputs.uniform_levels(7, 70 + C, (3, C, 11, 9), 4)
+    w = rng.standard_normal((40, C, ksz, ksz)).astype(np.float32)
+    acc_ref, out_ref, s_a, s_w = oracle.conv_layer(x, w, 4, 3, stride, pad, True, oracle.HTANH)
+    res = rng.standard_normal(out_ref.shape).astype(np.float32) * np.float32(0.5 * np.abs(out_ref).max())
+    xd, wd = _dev(x, cuda), _dev(w, cuda)
+    sa_d, sw_d = mpq.absmax(xd), mpq.absmax(wd, mpq.SCALE_PER_ROW)
+    xp = mpq.encode_nchw(xd, sa_d, 4)
+    wp, taps = mpq.encode_oihw(wd, sw_d, 3, mpq.SCALE_PER_ROW)
+    N, _, H, W = x.shape
+    yi = torch.empty(acc_ref.shape, dtype=torch.int32, device=cuda)
+    for residual, relu in ((None, False), (res, False), (res, True), (None, True)):
+        yf, yf_whole = _guarded(acc_ref.shape, torch.float32, cuda)
+        seen = mpq.zero(torch.full((1,), 7.0, dtype=torch.float32, device=cuda))
+        mpq.conv_fused(xp, 4, N, C, H, W, wp, 3, taps, 40, ksz, ksz, stride, pad, yi, yf, sa_d, sw_d,
+                       mpq.SCALE_PER_ROW, None if residual is None else _dev(residual, cuda), relu, seen)
+        ref = out_ref if residual is None else out_ref + residual
+        if relu:
+            ref = np.maximum(ref, np.float32(0))
+        assert np.array_equal(yi.cpu().numpy(), acc_ref)
+        assert np.array_equal(yf.cpu().numpy(), ref)                  # same single-rounded steps
+        assert _canaries_intact(yf_whole, acc_ref.size)
+        assert float(seen.cpu()[0]) == float(np.maximum(ref, 0).max())
+
+
+def test_maxpool_range(mpq, cuda):
+    x = np.random.default_rng(3).standard_normal((2, 5, 9, 12)).astype(np.float32)
+    seen = mpq.zero(torch.ones(1, dtype=torch.float32, device=cuda))
+    y = mpq.maxpool3x3s2(_dev(x, cuda), out_max=seen)
+    ref = torch.nn.functional.max_pool2d(torch.from_numpy(x), 3, 2, 1).numpy()
+    assert np.array_equal(y.cpu().numpy(), ref)
+    assert float(seen.cpu()[0]) == float(np.maximum(ref, 0).max())
+
+
 def test_conv_1x1_equals_gemm(mpq, cuda):
     """A 1x1 stride-1 convolution is the GEMM of the pixel matrix with the weight matrix."""
     x = inputs.uniform_levels(7, 1, (2, 128, 6, 5), 4)
