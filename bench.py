@@ -158,6 +158,25 @@ def _time_oracle(x, w, rows, steps, warmup):
     return tops, dt, oracle.threads(), sample
 
 
+def _oracle_other_workloads():
+    """CPU-baseline leg of --full: the oracle as it stands, timed once on workloads 1-3 in full
+    (range, quantize, integer product, scale).  Reported next to the GPU figures, never a target."""
+    import oracle
+    from paper_1905_13389_b200 import inputs
+    oracle.build()
+    out = {"cores": oracle.threads()}
+    c = inputs.config1()
+    t0 = time.perf_counter(); oracle.linear(c["x"], c["w"], 2, 2, a_act=oracle.HRELU); dt = time.perf_counter() - t0
+    out["gemm_w2a2_64x64x512"] = {"seconds": dt, "equivalent_tops": 2.0 * 64 * 64 * 512 / dt / 1e12}
+    c = inputs.config2()
+    t0 = time.perf_counter(); oracle.linear(c["x"], c["w"], 2, 2, w_per_row=True, a_act=oracle.HRELU); dt = time.perf_counter() - t0
+    out["fc_w2a2_64x4096x9216"] = {"seconds": dt, "equivalent_tops": 2.0 * c["m"] * c["n"] * c["k"] / dt / 1e12}
+    c = inputs.config3()
+    t0 = time.perf_counter(); oracle.conv_layer(c["x"], c["w"], 3, 3, 1, 1, True, oracle.HRELU); dt = time.perf_counter() - t0
+    out["conv3x3_w3a3_32x256x14x14"] = {"seconds": dt, "equivalent_tops": 2.0 * 6272 * 256 * 2304 / dt / 1e12}
+    return out
+
+
 def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
@@ -338,6 +357,12 @@ def run_cuda(args):
             del x, w, ap, wp, ci, cf, xh, wh, oi, of, ws
             torch.cuda.empty_cache()
             bench_suite.run_suite(dev, peaks["hbm_gbs"], args.full)
+            if not args.no_cpu_baseline:
+                with open(args.full) as fh:
+                    suite = json.load(fh)
+                suite["cpu_oracle"] = _oracle_other_workloads()
+                with open(args.full, "w") as fh:
+                    json.dump(suite, fh, indent=1)
     if world > 1:
         dist.destroy_process_group()
 
