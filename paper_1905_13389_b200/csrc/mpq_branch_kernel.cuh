@@ -479,7 +479,8 @@ static int launch_auto(const BranchParams& p, cudaStream_t st) {
     using T = BranchTile<HB, SB>;
     const int64_t held_tiles = ceil_div(p.held_rows, 16 * T::TH);
     const int64_t slots = 2 * 148;
-    const double penalty[3] = {1.00, 1.05, 1.20};      // TS = 8, 4, 2
+    // (with 7 or 8 streamed planes the 128-wide tile's loop body outgrows the instruction cache)
+    const double penalty[3] = {SB >= 7 ? 1.10 : 1.00, 1.05, 1.20};      // TS = 8, 4, 2
     int best = 0;
     double best_cost = 0.0;
     for (int c = 0; c < 3; ++c) {
