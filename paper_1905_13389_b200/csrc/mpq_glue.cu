@@ -7,77 +7,94 @@ namespace mpq {
 
 // ------------------------------------------------------------------------------------------
 // Stem: y[n][o][oh][ow] = relu?( sum_{c,kh,kw} x[n][c][2 oh + kh - 3][2 ow + kw - 3] * w[o][c][kh][kw] )
-// C = 3, O = 64, 7x7, stride 2, pad 3 (zero).  A CTA owns a 16 x 16 tile of output pixels of one
-// image: the 37 x 37 x 3 input patch and all 64 x 147 weights sit in shared memory; each thread
-// computes its pixel for 16 output channels at a time (weights read as broadcast 16-byte vectors).
-// Accumulation order per output: c, then kh, then kw, one fused multiply-add each.
+// C = 3, O = 64, 7x7, stride 2, pad 3 (zero).  A CTA owns 16 rows x 56 columns of output pixels of
+// one image (224 threads: 16 rows x 14 groups of 4 adjacent pixels); the 37 x 117 x 3 input patch
+// and all 64 x 147 weights sit in shared memory.  Per (c, kh) a thread reads the 13 inputs its four
+// pixels share and the weights of 16 output channels (broadcast 16-byte vectors) and issues
+// 7 x 4 x 16 fused multiply-adds from registers, so the loop is bound by the FP32 pipe, not by
+// shared-memory reads.  Accumulation order per output: c, then kh, then kw.
 // ------------------------------------------------------------------------------------------
-constexpr int kStemTile = 16;
-constexpr int kStemPatch = 2 * kStemTile + 5;      // 37
-constexpr int kStemTaps = 3 * 7 * 7;               // 147
+constexpr int kStemRows = 16;                       // output rows per CTA
+constexpr int kStemGroups = 14;                     // groups of 4 output columns per CTA
+constexpr int kStemCols = 4 * kStemGroups;          // 56
+constexpr int kStemThreads = kStemRows * kStemGroups;   // 224
+constexpr int kStemPatchH = 2 * kStemRows + 5;      // 37
+constexpr int kStemPatchW = 2 * kStemCols + 5;      // 117
+constexpr int kStemPatchStride = kStemPatchW + 1;   // 118
+constexpr int kStemTaps = 3 * 7 * 7;                // 147
 constexpr int kStemO = 64;
+constexpr int kStemWRow = 68;                      // floats per staged weight row (64 + 4: spreads the transposing stores over banks)
 
-__global__ void __launch_bounds__(kStemTile* kStemTile)
+__global__ void __launch_bounds__(kStemThreads)
 stem_conv7x7_kernel(const float* __restrict__ x, const float* __restrict__ w, float* __restrict__ y,
                     int N, int H, int W, int Ho, int Wo, int relu) {
     extern __shared__ __align__(16) float smem[];
     chain_entry();
-    float* ws = smem;                                   // [147][64]
-    float* xs = smem + kStemTaps * kStemO;              // [3][37][38]
-    constexpr int kRow = kStemPatch + 1;
+    float* ws = smem;                                   // [147][68]
+    float* xs = smem + kStemTaps * kStemWRow;           // [3][37][118]
     const int tid = threadIdx.x;
-    const int tiles_w = (Wo + kStemTile - 1) / kStemTile;
-    const int tiles_h = (Ho + kStemTile - 1) / kStemTile;
+    const int tiles_w = (Wo + kStemCols - 1) / kStemCols;
+    const int tiles_h = (Ho + kStemRows - 1) / kStemRows;
     const int n = blockIdx.x / (tiles_w * tiles_h);
     const int trem = blockIdx.x % (tiles_w * tiles_h);
-    const int oh0 = (trem / tiles_w) * kStemTile, ow0 = (trem % tiles_w) * kStemTile;
+    const int oh0 = (trem / tiles_w) * kStemRows, ow0 = (trem % tiles_w) * kStemCols;
 
-    for (int i = tid; i < kStemTaps * kStemO; i += blockDim.x) {
+    for (int i = tid; i < kStemTaps * kStemO; i += kStemThreads) {
         const int o = i / kStemTaps, t = i % kStemTaps;  // global order [o][c][kh][kw]
-        ws[t * kStemO + o] = __ldg(w + i);
+        ws[t * kStemWRow + o] = __ldg(w + i);
     }
     const int ih0 = oh0 * 2 - 3, iw0 = ow0 * 2 - 3;
-    for (int i = tid; i < 3 * kStemPatch * kStemPatch; i += blockDim.x) {
-        const int c = i / (kStemPatch * kStemPatch);
-        const int r = (i / kStemPatch) % kStemPatch, q = i % kStemPatch;
+    for (int i = tid; i < 3 * kStemPatchH * kStemPatchW; i += kStemThreads) {
+        const int c = i / (kStemPatchH * kStemPatchW);
+        const int r = (i / kStemPatchW) % kStemPatchH, q = i % kStemPatchW;
         const int ih = ih0 + r, iw = iw0 + q;
         float v = 0.0f;
         if (ih >= 0 && ih < H && iw >= 0 && iw < W) v = __ldg(x + (((int64_t)n * 3 + c) * H + ih) * W + iw);
-        xs[(c * kStemPatch + r) * kRow + q] = v;
+        xs[(c * kStemPatchH + r) * kStemPatchStride + q] = v;
     }
     __syncthreads();
 
-    const int ty = tid / kStemTile, tx = tid % kStemTile;
-    const int oh = oh0 + ty, ow = ow0 + tx;
-    const bool live = oh < Ho && ow < Wo;
+    const int ty = tid / kStemGroups, tg = tid % kStemGroups;
+    const int oh = oh0 + ty, ow = ow0 + 4 * tg;
     for (int o0 = 0; o0 < kStemO; o0 += 16) {
-        float acc[16];
+        float acc[4][16];
 #pragma unroll
-        for (int j = 0; j < 16; ++j) acc[j] = 0.0f;
+        for (int p = 0; p < 4; ++p)
+#pragma unroll
+            for (int j = 0; j < 16; ++j) acc[p][j] = 0.0f;
         for (int c = 0; c < 3; ++c) {
+#pragma unroll 1
             for (int kh = 0; kh < 7; ++kh) {
-                const float* xrow = xs + (c * kStemPatch + 2 * ty + kh) * kRow + 2 * tx;
-                const float* wrow = ws + ((c * 7 + kh) * 7) * kStemO + o0;
+                const float* xrow = xs + (c * kStemPatchH + 2 * ty + kh) * kStemPatchStride + 8 * tg;
+                float xv[13];
+#pragma unroll
+                for (int q = 0; q < 13; ++q) xv[q] = xrow[q];
+                const float* wrow = ws + ((c * 7 + kh) * 7) * kStemWRow + o0;
 #pragma unroll
                 for (int kw = 0; kw < 7; ++kw) {
-                    const float xv = xrow[kw];
-                    const float4* wv = reinterpret_cast<const float4*>(wrow + kw * kStemO);
+                    const float4* wv = reinterpret_cast<const float4*>(wrow + kw * kStemWRow);
 #pragma unroll
                     for (int q = 0; q < 4; ++q) {
                         const float4 f = wv[q];
-                        acc[4 * q + 0] = fmaf(xv, f.x, acc[4 * q + 0]);
-                        acc[4 * q + 1] = fmaf(xv, f.y, acc[4 * q + 1]);
-                        acc[4 * q + 2] = fmaf(xv, f.z, acc[4 * q + 2]);
-                        acc[4 * q + 3] = fmaf(xv, f.w, acc[4 * q + 3]);
+#pragma unroll
+                        for (int p = 0; p < 4; ++p) {
+                            const float xin = xv[2 * p + kw];
+                            acc[p][4 * q + 0] = fmaf(xin, f.x, acc[p][4 * q + 0]);
+                            acc[p][4 * q + 1] = fmaf(xin, f.y, acc[p][4 * q + 1]);
+                            acc[p][4 * q + 2] = fmaf(xin, f.z, acc[p][4 * q + 2]);
+                            acc[p][4 * q + 3] = fmaf(xin, f.w, acc[p][4 * q + 3]);
+                        }
                     }
                 }
             }
         }
-        if (live) {
+        if (oh < Ho) {
 #pragma unroll
             for (int j = 0; j < 16; ++j) {
-                const float v = relu ? fmaxf(acc[j], 0.0f) : acc[j];
-                y[(((int64_t)n * kStemO + o0 + j) * Ho + oh) * Wo + ow] = v;
+                float* dst = y + (((int64_t)n * kStemO + o0 + j) * Ho + oh) * Wo + ow;
+#pragma unroll
+                for (int p = 0; p < 4; ++p)
+                    if (ow + p < Wo) dst[p] = relu ? fmaxf(acc[p][j], 0.0f) : acc[p][j];
             }
         }
     }
@@ -123,9 +140,9 @@ extern "C" int mpq_stem_conv7x7(const float* x, const float* w, float* y, int N,
     if (!x || !w || !y) return MPQ_ERR_NULL;
     if (N <= 0 || H <= 0 || W <= 0) return MPQ_ERR_BAD_SHAPE;
     const int Ho = (H + 6 - 7) / 2 + 1, Wo = (W + 6 - 7) / 2 + 1;
-    const int64_t blocks = (int64_t)N * ceil_div(Ho, kStemTile) * ceil_div(Wo, kStemTile);
+    const int64_t blocks = (int64_t)N * ceil_div(Ho, kStemRows) * ceil_div(Wo, kStemCols);
     if (blocks > 0x7fffffffLL) return MPQ_ERR_BAD_SHAPE;
-    const size_t smem = (size_t)(kStemTaps * kStemO + 3 * kStemPatch * (kStemPatch + 1)) * sizeof(float);
+    const size_t smem = (size_t)(kStemTaps * kStemWRow + 3 * kStemPatchH * kStemPatchStride) * sizeof(float);
     static bool configured[64] = {};
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return MPQ_ERR_CUDA;
@@ -134,7 +151,7 @@ extern "C" int mpq_stem_conv7x7(const float* x, const float* w, float* y, int N,
             return MPQ_ERR_CUDA;
         configured[dev] = true;
     }
-    return launch_chained(stem_conv7x7_kernel, (unsigned)blocks, kStemTile * kStemTile, smem, (cudaStream_t)stream,
+    return launch_chained(stem_conv7x7_kernel, (unsigned)blocks, kStemThreads, smem, (cudaStream_t)stream,
                           x, w, y, N, H, W, Ho, Wo, relu);
 }
 
