@@ -64,7 +64,7 @@ int64_t mpq_row_words(int64_t k);
 /* Words of a whole packed operand: bits * rows * mpq_row_words(k).  0 on invalid arguments. */
 int64_t mpq_packed_words(int64_t rows, int64_t k, int bits);
 
-/* ---- Range.  BASELINE generalisation of the paper's fixed [-1,1] / [0,1] ranges (Table 1):
+/* ---- Range.  A generalisation of the paper's fixed [-1,1] / [0,1] ranges (Table 1) to data-dependent ones:
  * scale_out = max |x| (HTanh) or max of max(x,0) (HReLU), NaNs ignored; one value
  * (PER_TENSOR) or one per row (PER_ROW).  x is [rows x k] with row stride ldx (elements).
  * scale_out is overwritten (the call zeroes it first, on the stream). */
