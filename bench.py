@@ -357,12 +357,14 @@ def run_cuda(args):
             del x, w, ap, wp, ci, cf, xh, wh, oi, of, ws
             torch.cuda.empty_cache()
             bench_suite.run_suite(dev, peaks["hbm_gbs"], args.full)
+            with open(args.full) as fh:
+                suite = json.load(fh)
             if not args.no_cpu_baseline:
-                with open(args.full) as fh:
-                    suite = json.load(fh)
                 suite["cpu_oracle"] = _oracle_other_workloads()
                 with open(args.full, "w") as fh:
                     json.dump(suite, fh, indent=1)
+            with open(args.full + ".md", "w") as fh:
+                fh.write(bench_suite.summary_markdown(suite))
     if world > 1:
         dist.destroy_process_group()
 

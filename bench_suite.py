@@ -205,3 +205,51 @@ def run_suite(dev: torch.device, hbm_gbs: float, path: str):
     with open(path, "w") as fh:
         json.dump(out, fh, indent=1)
     return out
+
+
+def summary_markdown(d: dict) -> str:
+    """The suite's figures as the tables committed under profiles/."""
+    L = ["# Suite: all workloads on one B200 (`python bench.py --steps 20 --warmup 5 --full gpurun_out/suite.json`)\n",
+         "CUDA events on the launching stream after warm-up; short kernels replayed from a CUDA graph (no host launch",
+         "gaps).  Peaks measured in the same run: plain POPC pipe %.0f Gpopc/s, carry-save mix peak %.0f Gpopc/s"
+         % (d["popc_peak_gpopc_s"], d["branch_peak_gpopc_s"]),
+         "(probe at %.0f MHz), HBM copy %.0f GB/s (MEASURED_PEAKS.json).\n" % (d["probe_sm_mhz"], d["hbm_gbs"]),
+         "## Bit-width sweep, GEMM m = n = k = 4096, int32 out\n",
+         "| (w,a) bits | ms | equivalent TOPS | binary TOPS | frac of mix peak | frac of plain POPC pipe |",
+         "|---|---|---|---|---|---|"]
+    for k, r in d["gemm_sweep_4096"].items():
+        L.append("| %s | %.3f | %.1f | %.1f | %.3f | %.3f |" % (k, r["ms"], r["equivalent_tops"], r["binary_tops"],
+                                                             r["frac_of_branch_peak"], r["frac_of_plain_popc_peak"]))
+    L += ["\n## Other products\n", "| workload | time | equivalent TOPS | frac of mix peak | frac of plain POPC pipe |",
+          "|---|---|---|---|---|",
+          "| GEMM W2A2 64x64x512 (int32 + fp32 out) | %.1f us | launch-latency bound | – | – |" % d["gemm_w2a2_64x64x512"]["us"]]
+    r = d["fc_w2a2_64x4096x9216"]
+    L.append("| FC W2A2 64 x 4096 x 9216 (fp32 out, per-channel scale) | %.1f us | %.1f | %.3f | %.3f |"
+             % (r["ms"] * 1e3, r["equivalent_tops"], r["frac_of_branch_peak"], r["frac_of_plain_popc_peak"]))
+    r = d["conv3x3_w3a3_32x256x14x14"]
+    L.append("| conv 3x3 W3A3 32x256x14x14 -> 256 (fp32 out) | %.1f us (+ encode_nchw %.1f us) | %.1f | %.3f | %.3f |"
+             % (r["ms"] * 1e3, r["encode_nchw_us"], r["equivalent_tops"], r["frac_of_branch_peak"], r["frac_of_plain_popc_peak"]))
+    s = d["resnet18_stack_w4a4_b128"]
+    L += ["\n## ResNet-18-shaped stack, W4A4, batch 128, 224 x 224\n",
+          "%.2f ms per step = **%.0f images/s** end to end (fp32 stem + max-pool + 19 encoded convolutions; residual add,"
+          % (s["ms_per_step"], s["images_per_s"]),
+          "max(.,0) and every encoder's range ride in the producers' stores); encoded layers %.2f ms.  Span of an encoded"
+          % s["quantized_layers_ms"],
+          "layer = encode_nchw + conv (shortcut convolutions reuse conv1's planes).\n",
+          "| layer | ms | frac of mix peak | frac of plain POPC pipe |", "|---|---|---|---|"]
+    for n, r in s["layers"].items():
+        if "frac_of_branch_peak" in r:
+            L.append("| %s | %.3f | %.3f | %.3f |" % (n, r["ms"], r["frac_of_branch_peak"], r["frac_of_plain_popc_peak"]))
+        else:
+            L.append("| %s | %.3f | – | – |" % (n, r["ms"]))
+    L += ["\n## Encoders and range (HBM-bound)\n", "| kernel / tensor | us | GB/s | frac of measured copy bandwidth |", "|---|---|---|---|"]
+    for n, r in d["encoders"].items():
+        L.append("| %s | %.1f | %.0f | %.3f |" % (n, r["us"], r["gb_s"], r["frac_of_hbm"]))
+    if "cpu_oracle" in d:
+        o = d["cpu_oracle"]
+        L += ["\n## CPU oracle on the same host (%d cores), as it stands: a reported baseline, not a target\n" % o["cores"],
+              "| workload | seconds | equivalent TOPS |", "|---|---|---|"]
+        for n, r in o.items():
+            if isinstance(r, dict):
+                L.append("| %s | %.4f | %.4f |" % (n, r["seconds"], r["equivalent_tops"]))
+    return "\n".join(L) + "\n"
