@@ -57,6 +57,10 @@ def _load():
             lib.mpq_oracle_scale.restype = None
             lib.mpq_oracle_scale_f64.argtypes = [P, i64, i64, i64, f32, P, i32, i32, i32, P]
             lib.mpq_oracle_scale_f64.restype = None
+            lib.mpq_oracle_stem.argtypes = [P, P, i64, i64, i64, i32, P]
+            lib.mpq_oracle_stem.restype = None
+            lib.mpq_oracle_maxpool3x3s2.argtypes = [P, i64, i64, i64, P]
+            lib.mpq_oracle_maxpool3x3s2.restype = None
             _lib = lib
     return _lib
 
@@ -201,3 +205,24 @@ def conv_layer(x, w, a_bits: int, w_bits: int, stride: int = 1, pad: int = 0,
     qw = quantize(w, s_w, w_bits, per_row=w_per_channel)
     acc = conv(qx, qw, stride, pad)
     return acc, scale(acc, s_a[0], s_w, a_bits, w_bits), s_a, s_w
+
+
+def stem(x, w, relu: bool = True) -> np.ndarray:
+    """fp32 glue of the test network: 7x7 stride-2 pad-3 convolution, 3 -> 64 channels, each output one
+    chain of fused multiply-adds over (c, kh, kw); then max(.,0)."""
+    x, w = _f32c(x), _f32c(w)
+    N, C, H, W = x.shape
+    if C != 3 or w.shape != (64, 3, 7, 7):
+        raise ValueError("stem takes [N][3][H][W] and a [64][3][7][7] weight")
+    y = np.empty((N, 64, (H - 1) // 2 + 1, (W - 1) // 2 + 1), dtype=np.float32)
+    _load().mpq_oracle_stem(_p(x), _p(w), N, H, W, int(relu), _p(y))
+    return y
+
+
+def maxpool3x3s2(x) -> np.ndarray:
+    """3x3 max-pool, stride 2, pad 1 on [N][C][H][W]."""
+    x = _f32c(x)
+    N, C, H, W = x.shape
+    y = np.empty((N, C, (H - 1) // 2 + 1, (W - 1) // 2 + 1), dtype=np.float32)
+    _load().mpq_oracle_maxpool3x3s2(_p(x), N * C, H, W, _p(y))
+    return y

@@ -205,3 +205,49 @@ void mpq_oracle_scale_f64(const int32_t* acc, int64_t outer, int64_t channels, i
             }
         }
 }
+
+/* ---- Full-precision glue of the ResNet-shaped test network (not part of the paper's method;
+ * its first layer stays fp32).  Written out as the definition: a 7x7 stride-2 zero-padded
+ * convolution whose every output is one chain of fused multiply-adds over (c, kh, kw) in that
+ * order (fmaf is exactly rounded, so any implementation that keeps this order gives the same
+ * bits), then max(.,0); and a 3x3 stride-2 max-pool with padding 1. */
+void mpq_oracle_stem(const float* x, const float* w, int64_t N, int64_t H, int64_t W, int relu, float* y)
+{
+    const int64_t Ho = (H - 1) / 2 + 1, Wo = (W - 1) / 2 + 1;
+#pragma omp parallel for collapse(2) schedule(static)
+    for (int64_t n = 0; n < N; ++n)
+        for (int64_t o = 0; o < 64; ++o)
+            for (int64_t oh = 0; oh < Ho; ++oh)
+                for (int64_t ow = 0; ow < Wo; ++ow) {
+                    float acc = 0.0f;
+                    for (int64_t c = 0; c < 3; ++c)
+                        for (int64_t kh = 0; kh < 7; ++kh)
+                            for (int64_t kw = 0; kw < 7; ++kw) {
+                                const int64_t ih = 2 * oh + kh - 3, iw = 2 * ow + kw - 3;
+                                const float xv = (ih >= 0 && ih < H && iw >= 0 && iw < W)
+                                                     ? x[((n * 3 + c) * H + ih) * W + iw] : 0.0f;
+                                acc = fmaf(xv, w[((o * 3 + c) * 7 + kh) * 7 + kw], acc);
+                            }
+                    if (relu && !(acc > 0.0f)) acc = 0.0f;
+                    y[((n * 64 + o) * Ho + oh) * Wo + ow] = acc;
+                }
+}
+
+void mpq_oracle_maxpool3x3s2(const float* x, int64_t planes, int64_t H, int64_t W, float* y)
+{
+    const int64_t Ho = (H - 1) / 2 + 1, Wo = (W - 1) / 2 + 1;
+#pragma omp parallel for schedule(static)
+    for (int64_t p = 0; p < planes; ++p)
+        for (int64_t oh = 0; oh < Ho; ++oh)
+            for (int64_t ow = 0; ow < Wo; ++ow) {
+                float m = -INFINITY;
+                for (int64_t kh = 0; kh < 3; ++kh)
+                    for (int64_t kw = 0; kw < 3; ++kw) {
+                        const int64_t ih = 2 * oh + kh - 1, iw = 2 * ow + kw - 1;
+                        if (ih < 0 || ih >= H || iw < 0 || iw >= W) continue;
+                        const float v = x[(p * H + ih) * W + iw];
+                        if (v > m) m = v;
+                    }
+                y[(p * Ho + oh) * Wo + ow] = m;
+            }
+}

@@ -1,11 +1,12 @@
 """GPU parity of the ResNet-18-shaped stack of encoded convolutions (W4A4) against the CPU oracle.
 
-The fp32 stem is glue, checked against a float64 convolution; from the stem's pooled output on,
-the oracle runs the same chain of encoded layers (range -> quantize -> integer convolution ->
-scale, residual add + max in fp32) and every layer must agree: int32 accumulators bit-exact,
-fp32 outputs within 1e-5 relative.  The small case is compared element by element through the
-whole chain; the full-size case (batch 128, 224 x 224) on sampled outputs of every layer, each
-computed by the oracle from the GPU's own input to that layer.
+The oracle runs the whole network on its own from the raw input: the fp32 stem and max-pool (glue,
+defined as one fused-multiply-add chain per output, so bit-exact), then the chain of encoded layers
+(range -> quantize -> integer convolution -> scale, residual add + max in fp32); every layer must
+agree: int32 accumulators bit-exact, fp32 outputs within 1e-5 relative.  The small case is compared
+element by element through the whole chain.  At full size (batch 128, 224 x 224) the oracle cannot
+run the chain (2.2e11 multiply-adds), so the stem + max-pool are compared in full and every encoded
+layer on sampled outputs that the oracle computes one by one from that layer's input on the device.
 """
 import numpy as np
 import pytest
@@ -27,6 +28,7 @@ def test_stem_and_maxpool_against_float64(mpq, cuda):
     assert tuple(y.shape) == tuple(ref.shape) == (2, 64, 35, 35)
     err = (y.cpu().double() - ref).abs().max().item()
     assert err <= 1e-5 * ref.abs().max().item()            # 147-term fp32 sums against float64
+    assert np.array_equal(y.cpu().numpy(), oracle.stem(x, w, relu=False))   # same fma chain: same bits
     yr = mpq.stem_conv7x7(torch.from_numpy(x).to(cuda), torch.from_numpy(w).to(cuda), relu=True)
     assert torch.equal(yr, torch.clamp_min(y, 0))
     p = mpq.maxpool3x3s2(yr)
@@ -59,8 +61,9 @@ def test_stack_small_chain_elementwise(mpq, cuda, a_bits, w_bits, fused):
     net = QuantResNet18Stack(ws, batch, size, a_bits, w_bits, cuda, keep_int32=True, fused=fused)
     out = net.forward(torch.from_numpy(x).to(cuda))
     torch.cuda.synchronize()
-    cur = net.pooled.cpu().numpy()                         # the oracle chain starts from the stem's output
+    cur = oracle.maxpool3x3s2(oracle.stem(x, ws["conv1"]))  # the oracle's own chain, from the raw input
     assert cur.shape == (batch, 64, 16, 16) and cur.min() >= 0 and cur.max() > 0
+    assert np.array_equal(net.pooled.cpu().numpy(), cur)
     for blk, _, _, stride, has_ds in BLOCKS:
         res, cur = _oracle_block(cur, ws, blk, stride, has_ds, a_bits, w_bits)
         for name, (acc, ref) in res.items():
@@ -78,8 +81,10 @@ def test_stack_full_size_sampled(mpq, cuda):
     batch, size, a_bits, w_bits = 128, 224, 4, 4
     ws = inputs.config5_weights()
     net = QuantResNet18Stack(ws, batch, size, a_bits, w_bits, cuda, keep_int32=True, fused=True)
-    net.forward(torch.from_numpy(inputs.config5_input(batch, size)).to(cuda))
+    x = inputs.config5_input(batch, size)
+    net.forward(torch.from_numpy(x).to(cuda))
     torch.cuda.synchronize()
+    assert np.array_equal(net.pooled.cpu().numpy(), oracle.maxpool3x3s2(oracle.stem(x, ws["conv1"])))
     rng = np.random.default_rng(5)
     layer_in = net.pooled
     for blk, _, _, stride, has_ds in BLOCKS:
