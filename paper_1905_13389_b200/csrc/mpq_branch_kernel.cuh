@@ -275,28 +275,36 @@ branch_kernel(const BranchParams p) {
             }
         } else {
             // implicit im2col: one copy = `granule` words of one tap of one pixel (never crosses a tap).
-            // Index arithmetic is kept to shifts, compile-time divisors and one multiply-high.
+            // A thread owns one (pixel, k-quad) of the stage -- consecutive threads = consecutive
+            // pixels, which are contiguous in memory for a fixed tap -- works out the tap and its
+            // bounds once per copy position, and then only steps through the planes.  Index
+            // arithmetic is kept to shifts, compile-time divisors and one multiply-high.
             const int G = p.granule;
             const int gs = p.granule_shift;                 // copies per k-quad = 1 << gs
-            const int granules = S_QUADS << gs;
             const int64_t plane_words = (int64_t)p.N * p.H * p.W * p.Cw;
-            for (int id = tid; id < granules; id += 256) {
-                const int part = id & ((1 << gs) - 1);
-                const int q = id >> gs;
-                const int kq = q % KQ, row = (q / KQ) % BS, plane = q / (KQ * BS);
-                const uint32_t copy = (uint32_t)(((kq0 + kq) << gs) + part);   // copy index along k
-                const uint32_t tap = p.tap_granules == 1 ? copy : __umulhi(copy, p.tap_magic);
-                const int cw = (int)(copy - tap * p.tap_granules) * G;
-                const int kh = p.KW == 1 ? 0 : (int)((tap * 11u) >> 5);         // tap / 3 for tap < 9
-                const int kw = (int)tap - kh * p.KW;
-                const int ih = row_ih0[row] + kh, iw = row_iw0[row] + kw;
-                const bool ok = tap < (uint32_t)(p.KH * p.KW) && ih >= 0 && ih < p.H && iw >= 0 && iw < p.W;
-                const int pixel = row_pix[row] + kh * p.W + kw;
-                const uint32_t* src = ok ? p.streamed + plane * plane_words + (int64_t)pixel * p.Cw + cw : p.streamed;
-                uint32_t* dst = reinterpret_cast<uint32_t*>(ss + (plane * KQ + kq) * BS + row) + part * G;
-                if (G == 4) cp_async_16(dst, src, ok);
-                else if (G == 2) cp_async_small<8>(dst, src, ok);
-                else cp_async_small<4>(dst, src, ok);
+            constexpr int PS = (KQ * BS >= 256) ? 1 : (256 / (KQ * BS) < SB ? 256 / (KQ * BS) : SB);   // plane split
+            for (int item = tid; item < KQ * BS * PS; item += 256) {
+                const int row = item % BS, kq = (item / BS) % KQ, ps = item / (BS * KQ);
+                const int ih0 = row_ih0[row], iw0 = row_iw0[row], pix0 = row_pix[row];
+                for (int part = 0; part < (1 << gs); ++part) {
+                    const uint32_t copy = (uint32_t)(((kq0 + kq) << gs) + part);   // copy index along k
+                    const uint32_t tap = p.tap_granules == 1 ? copy : __umulhi(copy, p.tap_magic);
+                    const int cw = (int)(copy - tap * p.tap_granules) * G;
+                    const int kh = p.KW == 1 ? 0 : (int)((tap * 11u) >> 5);         // tap / 3 for tap < 9
+                    const int kw = (int)tap - kh * p.KW;
+                    const int ih = ih0 + kh, iw = iw0 + kw;
+                    const bool ok = tap < (uint32_t)(p.KH * p.KW) && ih >= 0 && ih < p.H && iw >= 0 && iw < p.W;
+                    const uint32_t* src = p.streamed + (ok ? (int64_t)(pix0 + kh * p.W + kw) * p.Cw + cw + ps * plane_words : 0);
+                    uint32_t* dst = reinterpret_cast<uint32_t*>(ss + (ps * KQ + kq) * BS + row) + part * G;
+#pragma unroll
+                    for (int plane = ps; plane < SB; plane += PS) {
+                        if (G == 4) cp_async_16(dst, src, ok);
+                        else if (G == 2) cp_async_small<8>(dst, src, ok);
+                        else cp_async_small<4>(dst, src, ok);
+                        if (ok) src += PS * plane_words;
+                        dst += PS * KQ * BS * 4;
+                    }
+                }
             }
         }
     };
