@@ -253,3 +253,43 @@ def summary_markdown(d: dict) -> str:
             if isinstance(r, dict):
                 L.append("| %s | %.4f | %.4f |" % (n, r["seconds"], r["equivalent_tops"]))
     return "\n".join(L) + "\n"
+
+
+def _single(argv):
+    """One product on its own, a few launches, for profiler captures:
+        python bench_suite.py gemm A_BITS W_BITS SIZE
+        python bench_suite.py conv BITS N C HW O KSIZE STRIDE
+    Prints the CUDA-event time of the last 10 launches."""
+    dev = torch.device("cuda:0")
+    torch.cuda.set_device(0)
+    if argv[0] == "gemm":
+        ab, wb, size = (int(a) for a in argv[1:4])
+        x = torch.randn(size, size, device=dev).relu_()
+        w = torch.randn(size, size, device=dev)
+        sa, sw = mpq.absmax(x), mpq.absmax(w)
+        ap, wp = mpq.encode(x, sa, ab), mpq.encode(w, sw, wb)
+        ci = torch.empty((size, size), dtype=torch.int32, device=dev)
+        fn = lambda: mpq.gemm(ap, ab, wp, wb, size, size, size, ci, None)
+        popcs = float(ab * wb) * size * size * (size // 32)
+    elif argv[0] == "conv":
+        bits, N, C, HW, O, ks, stride = (int(a) for a in argv[1:8])
+        x = torch.randn(N, C, HW, HW, device=dev).relu_()
+        w = torch.randn(O, C, ks, ks, device=dev)
+        sa, sw = mpq.absmax(x, 0, mpq.ACT_HRELU), mpq.absmax(w, mpq.SCALE_PER_ROW)
+        xp = mpq.encode_nchw(x, sa, bits, mpq.ACT_HRELU)
+        wp, taps = mpq.encode_oihw(w, sw, bits, mpq.SCALE_PER_ROW)
+        pad = ks // 2
+        Ho = (HW + 2 * pad - ks) // stride + 1
+        y = torch.empty((N, O, Ho, Ho), dtype=torch.float32, device=dev)
+        fn = lambda: mpq.conv(xp, bits, N, C, HW, HW, wp, bits, taps, O, ks, ks, stride, pad, None, y, sa, sw,
+                              mpq.SCALE_PER_ROW)
+        popcs = float(bits * bits) * N * Ho * Ho * O * (ks * ks * C // 32)
+    else:
+        raise SystemExit(_single.__doc__)
+    ms = _events_ms(fn, 10, 4)
+    print("%s: %.4f ms per launch, %.1f Gpopc/s" % (" ".join(argv), ms, popcs / (ms * 1e-3) / 1e9))
+
+
+if __name__ == "__main__":
+    import sys
+    _single(sys.argv[1:])
