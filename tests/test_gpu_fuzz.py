@@ -1,0 +1,68 @@
+"""Seeded random sweeps of the product kernels against the CPU oracle: shapes, bit-widths, strides
+and paddings drawn at random (every tile width, ragged tiles, short and half-filled k, single rows),
+all levels present in the operands.  int32 bit-exact, fp32 within 1e-5 relative."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_1905_13389_b200 import inputs
+from tests._util import rel_close
+
+pytestmark = pytest.mark.gpu
+
+
+def _dev(a, cuda):
+    return torch.from_numpy(np.ascontiguousarray(a)).to(cuda)
+
+
+@pytest.mark.parametrize("seed", range(24))
+def test_gemm_random_cases(mpq, cuda, seed):
+    rng = np.random.default_rng(1000 + seed)
+    a_bits, w_bits = int(rng.integers(1, 9)), int(rng.integers(1, 9))
+    m = int(rng.choice([1, 3, 17, 64, 65, 200, 513]))
+    n = int(rng.choice([1, 2, 31, 100, 128, 129, 700, 2500]))
+    k = int(rng.choice([1, 31, 32, 33, 127, 128, 129, 500, 1024, 3000]))
+    per_row = bool(rng.integers(0, 2))
+    act = int(rng.integers(0, 2))
+    x = inputs.uniform_levels(20, 2 * seed, (m, k), a_bits)
+    w = inputs.uniform_levels(20, 2 * seed + 1, (n, k), w_bits) * np.float32(0.5 + seed)
+    acc_ref, out_ref, s_a, s_w = oracle.linear(x, w, a_bits, w_bits, w_per_row=per_row, a_act=act)
+    xd, wd = _dev(x, cuda), _dev(w, cuda)
+    sa_d, sw_d = mpq.absmax(xd, 0, act), mpq.absmax(wd, int(per_row))
+    ap, wp = mpq.encode(xd, sa_d, a_bits, 0, act), mpq.encode(wd, sw_d, w_bits, int(per_row))
+    ci = torch.full((m, n), -5, dtype=torch.int32, device=cuda)
+    cf = torch.full((m, n), float("nan"), dtype=torch.float32, device=cuda)
+    mpq.gemm(ap, a_bits, wp, w_bits, m, n, k, ci, cf, sa_d, sw_d, int(per_row))
+    assert np.array_equal(ci.cpu().numpy(), acc_ref), (a_bits, w_bits, m, n, k)
+    assert rel_close(cf.cpu().numpy(), out_ref), (a_bits, w_bits, m, n, k)
+
+
+@pytest.mark.parametrize("seed", range(24))
+def test_conv_random_cases(mpq, cuda, seed):
+    rng = np.random.default_rng(2000 + seed)
+    a_bits, w_bits = int(rng.integers(1, 9)), int(rng.integers(1, 9))
+    C = int(rng.choice([32, 64, 128, 256, 384]))
+    ksz = int(rng.choice([1, 3]))
+    stride = int(rng.choice([1, 2]))
+    pad = int(rng.integers(0, 2)) if ksz == 3 else 0
+    H = int(rng.integers(3, 20))
+    W = int(rng.integers(3, 20))
+    N = int(rng.choice([1, 2, 5, 9]))
+    O = int(rng.choice([1, 7, 32, 33, 80]))
+    if a_bits + w_bits > 12 and C > 128:          # keep 9 * C * L_a * L_w inside int32
+        C = 128
+    act = int(rng.integers(0, 2))
+    x = inputs.uniform_levels(21, 2 * seed, (N, C, H, W), a_bits)
+    w = inputs.uniform_levels(21, 2 * seed + 1, (O, C, ksz, ksz), w_bits)
+    acc_ref, out_ref, s_a, s_w = oracle.conv_layer(x, w, a_bits, w_bits, stride, pad, True, act)
+    xd, wd = _dev(x, cuda), _dev(w, cuda)
+    sa_d, sw_d = mpq.absmax(xd, 0, act), mpq.absmax(wd, mpq.SCALE_PER_ROW)
+    xp = mpq.encode_nchw(xd, sa_d, a_bits, act)
+    wp, taps = mpq.encode_oihw(wd, sw_d, w_bits, mpq.SCALE_PER_ROW)
+    yi = torch.full(acc_ref.shape, -5, dtype=torch.int32, device=cuda)
+    yf = torch.full(acc_ref.shape, float("nan"), dtype=torch.float32, device=cuda)
+    mpq.conv(xp, a_bits, N, C, H, W, wp, w_bits, taps, O, ksz, ksz, stride, pad, yi, yf, sa_d, sw_d, mpq.SCALE_PER_ROW)
+    key = (a_bits, w_bits, N, C, H, W, O, ksz, stride, pad)
+    assert np.array_equal(yi.cpu().numpy(), acc_ref), key
+    assert rel_close(yf.cpu().numpy(), out_ref), key
