@@ -6,9 +6,9 @@
 //     S[r][c] = sum_{i,j} 2^(i+j) * popcount(A_i[r] xor B_j[c])
 // for a small register tile of outputs, then applies the decoder
 //     acc = L_a L_w k - 2 S,   out = float(acc) * alpha[c]           (Eq. 18)
-// in the store.  The arithmetic is XOR + POPC + shift-add on the integer pipes: the B200's
-// 5th-generation tensor cores have no 1-bit kind, and the legacy 1-bit mma.sync form measured
-// slower than the POPC pipe on this chip.
+// in the store.  The arithmetic is XOR, bitwise full adders (carry-save) and POPC on the integer
+// pipes, with the weighted adds as integer multiply-adds: the B200's 5th-generation tensor cores
+// have no 1-bit kind, and the legacy 1-bit mma.sync form measured slower than this path.
 //
 // Roles.  The "held" operand (HB planes, TH items per thread) lives in registers as 128-bit
 // k-quads; the "streamed" operand (SB planes, TS items per thread) is read quad by quad from
