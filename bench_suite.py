@@ -87,6 +87,18 @@ def run_suite(dev: torch.device, hbm_gbs: float, path: str):
         sweep["w%da%d" % (w_bits, a_bits)] = product_record(ms, size, size, size, a_bits, w_bits,
                                                              float(a_bits * w_bits) * size * size * (size // 32))
     out["gemm_sweep_4096"] = sweep
+    # context only, not this path: what a library int8 tensor-core GEMM of the same shape costs
+    # (the product of the DECODED integers, which fit int8 up to 7 bits; cuBLASLt through torch)
+    try:
+        qa = torch.randint(-3, 4, (size, size), dtype=torch.int8, device=dev)
+        qb = torch.randint(-3, 4, (size, size), dtype=torch.int8, device=dev)
+        ms = _events_ms(lambda: torch._int_mm(qa, qb), 10, 3)
+        out["context_library_int8_gemm_4096"] = {"ms": ms, "tops": 2.0 * size ** 3 / (ms * 1e-3) / 1e12,
+                                                 "note": "decoded-integer product on the tensor cores (library kernel); "
+                                                         "not the bit-plane path and not part of this library"}
+        del qa, qb
+    except Exception as exc:                                    # library kernel unavailable: the context line is dropped
+        out["context_library_int8_gemm_4096"] = {"unavailable": str(exc)[:200]}
 
     # ---- encoders on the sweep's operands (64 MiB fp32 each; four buffers in rotation) ----------
     xs = [x, w, torch.randn_like(x), torch.randn_like(x)]
@@ -220,6 +232,10 @@ def summary_markdown(d: dict) -> str:
     for k, r in d["gemm_sweep_4096"].items():
         L.append("| %s | %.3f | %.1f | %.1f | %.3f | %.3f |" % (k, r["ms"], r["equivalent_tops"], r["binary_tops"],
                                                              r["frac_of_branch_peak"], r["frac_of_plain_popc_peak"]))
+    ctx = d.get("context_library_int8_gemm_4096", {})
+    if "ms" in ctx:
+        L.append("\nContext only (not this path): a library int8 tensor-core GEMM of the decoded integers, same shape: "
+                 "%.3f ms = %.0f TOPS." % (ctx["ms"], ctx["tops"]))
     L += ["\n## Other products\n", "| workload | time | equivalent TOPS | frac of mix peak | frac of plain POPC pipe |",
           "|---|---|---|---|---|",
           "| GEMM W2A2 64x64x512 (int32 + fp32 out) | %.1f us | launch-latency bound | – | – |" % d["gemm_w2a2_64x64x512"]["us"]]

@@ -217,6 +217,27 @@ def test_gemm_extreme_codes_int32_headroom(mpq, cuda, a_bits, w_bits, k):
     assert abs(int(ref[0, 1])) == k * La * Lw
 
 
+@pytest.mark.parametrize("a_bits,w_bits", [(2, 2), (4, 3), (7, 7)])
+def test_gemm_equals_library_int8_product_of_decoded_integers(mpq, cuda, a_bits, w_bits):
+    """Eq. 7-10 as a whole: the branch-decomposed product on bit-planes equals the plain integer
+    product of the decoded odd integers, here computed by a library int8 GEMM on the device
+    (an independent route; the integers come from the CPU oracle's quantizer)."""
+    if not hasattr(torch, "_int_mm"):
+        pytest.skip("no library int8 GEMM in this torch")
+    m, n, k = 64, 96, 256
+    x = inputs.uniform_levels(9, 40 + a_bits, (m, k), a_bits)
+    w = inputs.uniform_levels(9, 50 + w_bits, (n, k), w_bits)
+    one = _dev(np.ones(1, np.float32), cuda)
+    qa = oracle.quantize(x, 1.0, a_bits).astype(np.int8)
+    qb = oracle.quantize(w, 1.0, w_bits).astype(np.int8)
+    ref = torch._int_mm(_dev(qa, cuda), _dev(np.ascontiguousarray(qb.T), cuda))
+    ci = torch.empty((m, n), dtype=torch.int32, device=cuda)
+    mpq.gemm(mpq.encode(_dev(x, cuda), one, a_bits), a_bits, mpq.encode(_dev(w, cuda), one, w_bits), w_bits,
+             m, n, k, ci, None)
+    assert torch.equal(ci, ref)
+    assert np.array_equal(ci.cpu().numpy(), oracle.gemm(qa.astype(np.int16), qb.astype(np.int16)))
+
+
 def test_gemm_config2_fc(mpq, cuda):
     c = inputs.config2()
     _gemm_case(mpq, cuda, c["x"], c["w"], 2, 2, w_per_row=True, both=False)
