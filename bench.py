@@ -321,7 +321,7 @@ def run_cuda(args):
             "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "int32", "data": "synthetic",
             "config": dict(_config(), binary_tops=value * A_BITS * W_BITS),
-            "roofline": {"bound": "alu", "kernel": "branch_kernel<2,2,8,gemm> (XOR + carry-save + POPC GEMM)",
+            "roofline": {"bound": "alu", "kernel": "branch_kernel<2,2,4,gemm> (XOR + carry-save + POPC GEMM, 64 x 64 tile, 3 CTAs per SM)",
                          "achieved": achieved / 1e9, "peak": branch_peak / 1e9, "unit": "Gpopc/s",
                          "frac": achieved / branch_peak, "traffic": GEMM_DRAM_TRAFFIC_BYTES,
                          "peak_source": "measured live at %.0f MHz on %d SMs: issue rate of the carry-save instruction mix "

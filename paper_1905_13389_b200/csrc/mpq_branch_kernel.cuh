@@ -191,10 +191,14 @@ struct BranchTile {
     // the k-quads of a stage are unrolled only while the loop body stays small enough for the
     // instruction cache (about 12 instructions per plane pair per output)
     static constexpr bool UNROLL_KQ = HB * SB <= 4;
+    // CTAs per SM: the 64-wide tile (TS = 4) fits three times with 80 registers per thread as long
+    // as the product has at most 16 plane pairs; a third resident CTA gives the two integer pipes
+    // more warps to interleave (W4A4: 0.92 -> 0.94 of the instruction-mix peak).
+    static constexpr int resident(int ts) { return (ts == 4 && HB * SB <= 16) ? 3 : 2; }
 };
 
 template <int HB, int SB, int TS, int MODE>
-__global__ void __launch_bounds__(256, 2)
+__global__ void __launch_bounds__(256, BranchTile<HB, SB>::resident(TS))
 branch_kernel(const BranchParams p) {
     using T = BranchTile<HB, SB>;
     constexpr int TH = T::TH, KQ = T::KQ, STAGES = T::STAGES;
@@ -480,21 +484,25 @@ static int launch_branch(const BranchParams& p, cudaStream_t st) {
 
 // Streamed-side tile width (16*TS items): the widest tile has the least shared-memory traffic per
 // population count, but a grid of few large tiles leaves SMs idle in its last wave.  Pick the
-// width with the smallest estimated makespan: waves of (2 CTAs x 148 SMs) tiles, each costing
-// its width times a measured per-width inefficiency.
+// width with the smallest estimated makespan: waves of (resident CTAs x 148 SMs) tiles, each
+// costing its width times the CTAs that share an SM times a measured per-width inefficiency.
 template <int HB, int SB, int MODE>
 static int launch_auto(const BranchParams& p, cudaStream_t st) {
     using T = BranchTile<HB, SB>;
     const int64_t held_tiles = ceil_div(p.held_rows, 16 * T::TH);
-    const int64_t slots = 2 * 148;
     // (with 7 or 8 streamed planes the 128-wide tile's loop body outgrows the instruction cache)
-    const double penalty[3] = {SB >= 7 ? 1.10 : 1.00, 1.05, 1.20};      // TS = 8, 4, 2
+    const double penalty[3] = {SB >= 7 ? 1.10 : 1.00, T::resident(4) == 3 ? 0.98 : 1.05, 1.20};      // TS = 8, 4, 2
     int best = 0;
     double best_cost = 0.0;
     for (int c = 0; c < 3; ++c) {
         const int ts = 8 >> c;
+        const int per_sm = T::resident(ts);
+        const int64_t slots = (int64_t)per_sm * 148;
         const int64_t tiles = ceil_div(p.streamed_rows, 16 * ts) * held_tiles;
-        const double cost = (double)ceil_div(tiles, slots) * ts * penalty[c];
+        // a grid that fits the resident slots takes one tile time; a longer one its share of waves
+        // plus half a wave of tail; a tile's time grows with its width and with the CTAs sharing the SM
+        const double waves = tiles <= slots ? 1.0 : (double)tiles / (double)slots + 0.5;
+        const double cost = waves * ts * per_sm * penalty[c];
         if (c == 0 || cost < best_cost) { best = c; best_cost = cost; }
     }
     if (best == 0) return launch_branch<HB, SB, 8, MODE>(p, st);
