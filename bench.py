@@ -34,9 +34,9 @@ SIZE = 4096
 A_BITS = W_BITS = 2
 HBM_FALLBACK_GBS = 6650.0      # used only when MEASURED_PEAKS.json is absent
 # DRAM bytes per launch of the GEMM kernel (dram__bytes_read.sum + dram__bytes_write.sum) from the
-# committed ncu capture of this command, profiles/branch_kernel_w2a2_gemm4096.md: 8.68 MB + 81.15 MB.
+# committed ncu capture of this command, profiles/branch_kernel_w2a2_gemm4096.md: 8.46 MB + 80.40 MB.
 # Set back to None whenever branch_kernel changes after that capture.
-GEMM_DRAM_TRAFFIC_BYTES = 89.8e6
+GEMM_DRAM_TRAFFIC_BYTES = 88.9e6
 
 
 def _peaks():
