@@ -332,7 +332,8 @@ def run_cuda(args):
                                              "lanes_per_clk_per_sm": popc_peak / (probe_mhz * 1e6 * sms),
                                              "note": "one POPC per xor word (no carry-save) cannot exceed this; the "
                                                      "kernel issues half as many POPCs as algorithmic popcounts"},
-                         "ms_per_launch": gemm_ms, "algorithmic_popc_per_launch": popcs},
+                         "ms_per_launch": gemm_ms, "algorithmic_popc_per_launch": popcs,
+                         "equivalent_tops_of_this_kernel": 2.0 * m * n * k / (gemm_ms * 1e-3) / 1e12},
             "encode": {"bound": "hbm", "achieved": enc_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                        "frac": enc_gbs / peaks["hbm_gbs"], "peak_source": "%s copy bandwidth" % peak_kind,
                        "ms_per_step": enc_ms, "bytes_per_step": enc_bytes,
