@@ -238,6 +238,40 @@ def test_gemm_equals_library_int8_product_of_decoded_integers(mpq, cuda, a_bits,
     assert np.array_equal(ci.cpu().numpy(), oracle.gemm(qa.astype(np.int16), qb.astype(np.int16)))
 
 
+@pytest.mark.parametrize("pad_in,pad_out", [(4, 5), (1, 0), (0, 3)])
+def test_strided_rows_through_the_c_abi(mpq, cuda, pad_in, pad_out):
+    """Row strides larger than the row length (ldx > k for range and encode, ldc > n for the product),
+    which the binding never passes: straight through the C entry points."""
+    m, n, k = 21, 37, 2100
+    rng = np.random.default_rng(pad_in * 7 + pad_out)
+    xw = rng.standard_normal((m, k + pad_in)).astype(np.float32)
+    ww = rng.standard_normal((n, k + pad_in)).astype(np.float32)
+    xw[:, k:] = 1e9; ww[:, k:] = -1e9                      # poison outside the rows: must never be read as data
+    x, w = np.ascontiguousarray(xw[:, :k]), np.ascontiguousarray(ww[:, :k])
+    acc_ref, out_ref, s_a, s_w = oracle.linear(x, w, 3, 2, w_per_row=True)
+    L = mpq.lib()
+    xd, wd = _dev(xw, cuda), _dev(ww, cuda)
+    sa = torch.empty(1, dtype=torch.float32, device=cuda)
+    sw = torch.empty(n, dtype=torch.float32, device=cuda)
+    st = torch.cuda.current_stream().cuda_stream
+    assert L.mpq_absmax(xd.data_ptr(), m, k, k + pad_in, 0, 0, sa.data_ptr(), st) == 0
+    assert L.mpq_absmax(wd.data_ptr(), n, k, k + pad_in, 1, 0, sw.data_ptr(), st) == 0
+    assert np.array_equal(sa.cpu().numpy(), s_a) and np.array_equal(sw.cpu().numpy(), s_w)
+    rw = mpq.row_words(k)
+    ap = torch.empty((3, m, rw), dtype=torch.int32, device=cuda)
+    wp = torch.empty((2, n, rw), dtype=torch.int32, device=cuda)
+    assert L.mpq_encode(xd.data_ptr(), m, k, k + pad_in, sa.data_ptr(), 0, 0, 3, ap.data_ptr(), st) == 0
+    assert L.mpq_encode(wd.data_ptr(), n, k, k + pad_in, sw.data_ptr(), 1, 0, 2, wp.data_ptr(), st) == 0
+    ldc = n + pad_out
+    ci = torch.full((m, ldc), 12345, dtype=torch.int32, device=cuda)
+    cf = torch.full((m, ldc), 7.0, dtype=torch.float32, device=cuda)
+    assert L.mpq_gemm(ap.data_ptr(), 3, wp.data_ptr(), 2, m, n, k, ci.data_ptr(), cf.data_ptr(), ldc,
+                      sa.data_ptr(), sw.data_ptr(), 1, st) == 0
+    assert np.array_equal(ci[:, :n].cpu().numpy(), acc_ref)
+    assert rel_close(cf[:, :n].cpu().numpy(), out_ref)
+    assert bool((ci[:, n:] == 12345).all()) and bool((cf[:, n:] == 7.0).all())     # the gap between rows is untouched
+
+
 def test_gemm_config2_fc(mpq, cuda):
     c = inputs.config2()
     _gemm_case(mpq, cuda, c["x"], c["w"], 2, 2, w_per_row=True, both=False)
