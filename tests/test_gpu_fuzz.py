@@ -66,3 +66,19 @@ def test_conv_random_cases(mpq, cuda, seed):
     key = (a_bits, w_bits, N, C, H, W, O, ksz, stride, pad)
     assert np.array_equal(yi.cpu().numpy(), acc_ref), key
     assert rel_close(yf.cpu().numpy(), out_ref), key
+
+
+def test_gemm_very_tall_and_very_wide(mpq, cuda):
+    """Grid extremes: 200 000 rows against a handful of columns, and the transpose of that shape."""
+    for (m, n) in ((200000, 5), (5, 200000)):
+        k = 96
+        x = inputs.uniform_levels(22, m % 7, (m, k), 2)
+        w = inputs.uniform_levels(22, 10 + n % 7, (n, k), 3)
+        acc_ref, out_ref, s_a, s_w = oracle.linear(x, w, 2, 3, w_per_row=False)
+        xd, wd = _dev(x, cuda), _dev(w, cuda)
+        sa_d, sw_d = mpq.absmax(xd), mpq.absmax(wd)
+        ci = torch.empty((m, n), dtype=torch.int32, device=cuda)
+        cf = torch.empty((m, n), dtype=torch.float32, device=cuda)
+        mpq.gemm(mpq.encode(xd, sa_d, 2), 2, mpq.encode(wd, sw_d, 3), 3, m, n, k, ci, cf, sa_d, sw_d)
+        assert np.array_equal(ci.cpu().numpy(), acc_ref)
+        assert rel_close(cf.cpu().numpy(), out_ref)
