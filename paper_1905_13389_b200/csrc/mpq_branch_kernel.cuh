@@ -190,7 +190,7 @@ struct BranchTile {
     static constexpr int CSA_BUDGET = 2 * HB * SB * GQ;
     // the k-quads of a stage are unrolled only while the loop body stays small enough for the
     // instruction cache (about 12 instructions per plane pair per output)
-    static constexpr bool UNROLL_KQ = HB * SB <= 4;
+    static constexpr bool UNROLL_KQ = HB * SB <= 9;
     // CTAs per SM: the 64-wide tile (TS = 4) fits three times with 80 registers per thread as long
     // as the product has at most 16 plane pairs; a third resident CTA gives the two integer pipes
     // more warps to interleave (W4A4: 0.92 -> 0.94 of the instruction-mix peak).
