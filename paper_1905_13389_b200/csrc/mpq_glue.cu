@@ -101,28 +101,44 @@ stem_conv7x7_kernel(const float* __restrict__ x, const float* __restrict__ w, fl
 }
 
 // 3x3 max-pool, stride 2, pad 1 (padding never wins: the window always holds a real element).
+// A thread produces four adjacent outputs of a row from the 3 x 9 inputs they share, so that
+// 27 loads are in flight per thread and neighbouring threads read neighbouring columns.
 __global__ void maxpool3x3s2_kernel(const float* __restrict__ x, float* __restrict__ y,
                                     int64_t planes, int H, int W, int Ho, int Wo, float* out_max) {
     chain_entry();
     float seen_max = 0.0f;
-    const int64_t total = planes * Ho * Wo;
+    const int groups = (Wo + 3) / 4;                       // groups of 4 outputs per row
+    const int64_t total = planes * Ho * groups;
     const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    const float ninf = -__int_as_float(0x7f800000);
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += stride) {
-        const int ow = (int)(i % Wo), oh = (int)((i / Wo) % Ho);
-        const int64_t pl = i / ((int64_t)Wo * Ho);
+        const int g = (int)(i % groups), oh = (int)((i / groups) % Ho);
+        const int64_t pl = i / ((int64_t)groups * Ho);
         const float* xp = x + pl * H * W;
-        float m = -__int_as_float(0x7f800000);
+        const int ow0 = 4 * g, iw0 = 2 * ow0 - 1;
+        float col[9];                                      // column maxima over the three rows
+#pragma unroll
+        for (int q = 0; q < 9; ++q) col[q] = ninf;
+#pragma unroll
         for (int kh = 0; kh < 3; ++kh) {
             const int ih = 2 * oh + kh - 1;
             if (ih < 0 || ih >= H) continue;
-            for (int kw = 0; kw < 3; ++kw) {
-                const int iw = 2 * ow + kw - 1;
-                if (iw < 0 || iw >= W) continue;
-                m = fmaxf(m, __ldg(xp + (int64_t)ih * W + iw));
+            const float* row = xp + (int64_t)ih * W;
+#pragma unroll
+            for (int q = 0; q < 9; ++q) {
+                const int iw = iw0 + q;
+                if (iw >= 0 && iw < W) col[q] = fmaxf(col[q], __ldg(row + iw));
             }
         }
-        y[i] = m;
-        seen_max = fmaxf(seen_max, m);
+        float* dst = y + (pl * Ho + oh) * Wo + ow0;
+#pragma unroll
+        for (int t = 0; t < 4; ++t) {
+            if (ow0 + t < Wo) {
+                const float m = fmaxf(fmaxf(col[2 * t], col[2 * t + 1]), col[2 * t + 2]);
+                dst[t] = m;
+                seen_max = fmaxf(seen_max, m);
+            }
+        }
     }
     if (out_max) {
 #pragma unroll
@@ -160,8 +176,8 @@ extern "C" int mpq_maxpool3x3s2(const float* x, float* y, int N, int C, int H, i
     if (!x || !y) return MPQ_ERR_NULL;
     if (N <= 0 || C <= 0 || H <= 0 || W <= 0) return MPQ_ERR_BAD_SHAPE;
     const int Ho = (H + 2 - 3) / 2 + 1, Wo = (W + 2 - 3) / 2 + 1;
-    const int64_t total = (int64_t)N * C * Ho * Wo;
-    const int64_t blocks = min((int64_t)148 * 16, ceil_div(total, 256));
+    const int64_t total = (int64_t)N * C * Ho * ((Wo + 3) / 4);
+    const int64_t blocks = min((int64_t)148 * 32, ceil_div(total, 256));
     return launch_chained(maxpool3x3s2_kernel, (unsigned)blocks, 256, 0, (cudaStream_t)stream,
                           x, y, (int64_t)N * C, H, W, Ho, Wo, out_max);
 }
