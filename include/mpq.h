@@ -11,8 +11,10 @@
  *
  * Conventions for every entry point
  *   - Pointers are DEVICE pointers unless the name ends in _host.  The caller owns and
- *     sizes every buffer; the library allocates nothing and keeps no state between calls
- *     (mpq_linear and mpq_linear_host stage through a caller-provided device workspace).
+ *     sizes every buffer; the library allocates no device memory and keeps no state between
+ *     calls (mpq_linear and mpq_linear_host stage through a caller-provided device workspace).
+ *     Two documented exceptions: mpq_linear_static works on a buffer built into the library
+ *     image, and mpq_linear_host keeps one helper stream and a few events per device.
  *   - Calls are asynchronous on `stream` (a cudaStream_t passed as void*; NULL = the
  *     default stream) unless stated otherwise.  Outputs are fully overwritten.
  *   - Return value: an mpq_status.  Errors that the host can see (null pointers, bad
