@@ -112,6 +112,23 @@ def test_encode_rows_full_segments_with_specials(mpq, cuda, bits):
             assert np.array_equal(u, oracle.levels(oracle.quantize(x, s, bits, act=act), bits))
 
 
+@pytest.mark.parametrize("bits,act", [(2, 0), (3, 1), (8, 0)])
+def test_encode_every_float_of_a_binade(mpq, cuda, bits, act):
+    """Every float32 with |x| in [1/2, 1) -- 16.8 million inputs, all level boundaries of the upper half
+    of the range with their neighbours -- against the oracle's quantizer, plane by plane.  (The same
+    comparison over all 2^32 bit patterns was run once when the FMA-pipe quantizer was written.)"""
+    lo, hi = np.float32(0.5).view(np.uint32), np.float32(1.0).view(np.uint32)
+    pos = np.arange(lo, hi, dtype=np.uint32)
+    k = 1 << 20
+    x = np.concatenate([pos, pos | np.uint32(0x80000000)]).view(np.float32).reshape(-1, k)
+    one = _dev(np.ones(1, np.float32), cuda)
+    planes = mpq.encode(_dev(x, cuda), one, bits, 0, act).cpu().numpy().view(np.uint32)
+    u = oracle.levels(oracle.quantize(x, 1.0, bits, act=act), bits)
+    for p in range(bits):
+        ref = np.packbits(((u >> p) & 1).astype(np.uint8), axis=1, bitorder="little").view(np.uint32)
+        assert np.array_equal(ref, planes[p]), p
+
+
 @pytest.mark.parametrize("bits", [1, 2, 3, 4, 8])
 @pytest.mark.parametrize("shape", [(2, 32, 5, 7), (1, 64, 9, 9), (3, 128, 4, 6), (2, 256, 14, 14)])
 def test_encode_nchw_codes(mpq, cuda, bits, shape):
