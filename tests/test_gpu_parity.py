@@ -129,6 +129,19 @@ def test_encode_every_float_of_a_binade(mpq, cuda, bits, act):
         assert np.array_equal(ref, planes[p]), p
 
 
+def test_encode_nchw_every_float_of_a_binade(mpq, cuda):
+    """The same 16.8 million inputs through the NCHW encoder (4 bits, HReLU), word by word."""
+    lo, hi = np.float32(0.5).view(np.uint32), np.float32(1.0).view(np.uint32)
+    pos = np.arange(lo, hi, dtype=np.uint32)
+    x = np.concatenate([pos, pos | np.uint32(0x80000000)]).view(np.float32).reshape(16, 64, 128, 128)
+    one = _dev(np.ones(1, np.float32), cuda)
+    planes = mpq.encode_nchw(_dev(x, cuda), one, 4, mpq.ACT_HRELU).cpu().numpy().view(np.uint32)   # [4][N][H][W][2]
+    u = oracle.levels(oracle.quantize(x, 1.0, 4, act=oracle.HRELU), 4).transpose(0, 2, 3, 1)       # [N][H][W][C]
+    for p in range(4):
+        ref = np.packbits(((u >> p) & 1).astype(np.uint8), axis=3, bitorder="little").view(np.uint32)
+        assert np.array_equal(ref.reshape(planes[p].shape), planes[p]), p
+
+
 @pytest.mark.parametrize("bits", [1, 2, 3, 4, 8])
 @pytest.mark.parametrize("shape", [(2, 32, 5, 7), (1, 64, 9, 9), (3, 128, 4, 6), (2, 256, 14, 14)])
 def test_encode_nchw_codes(mpq, cuda, bits, shape):
