@@ -436,10 +436,11 @@ branch_kernel(const BranchParams p) {
                 if (o >= p.held_rows) continue;
                 int32_t v = (int32_t)(full - 2u * acc[a][b]);
                 if (outside) {
-                    int32_t fix = 0;
+                    // modular arithmetic: the staged value may leave the int32 range, the corrected one does not
+                    uint32_t fix = 0u;
                     for (int t = 0; t < taps; ++t)
-                        if (outside & (1u << t)) fix += __ldg(p.tap_sums + (int64_t)t * p.O + o);
-                    v += ((1 << A_BITS) - 1) * fix;
+                        if (outside & (1u << t)) fix += (uint32_t)__ldg(p.tap_sums + (int64_t)t * p.O + o);
+                    v = (int32_t)((uint32_t)v + (uint32_t)((1 << A_BITS) - 1) * fix);
                 }
                 const int64_t idx = ((int64_t)n * p.O + o) * hw + rem;
                 if (p.out_i32) p.out_i32[idx] = v;

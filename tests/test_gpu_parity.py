@@ -417,6 +417,28 @@ def test_maxpool_range(mpq, cuda):
     assert float(seen.cpu()[0]) == float(np.maximum(ref, 0).max())
 
 
+def test_conv_extreme_codes_int32_headroom(mpq, cuda):
+    """All-extreme 8-bit codes at the largest channel count the int32 contract allows for a 3x3 filter
+    (9 * 3584 * 255 * 255 = 2.10e9 < 2^31), with zero padding: interior outputs sit at -k L_a L_w and the
+    border correction works on values whose staged form leaves the int32 range."""
+    C, O = 3584, 3
+    x = np.ones((1, C, 4, 4), np.float32)
+    w = -np.ones((O, C, 3, 3), np.float32)
+    w[1] = 1.0
+    w[2, ::2] = 1.0
+    acc_ref, out_ref, s_a, s_w = oracle.conv_layer(x, w, 8, 8, 1, 1, True, oracle.HTANH)
+    assert int(acc_ref[0, 0, 1, 1]) == -9 * C * 255 * 255 and int(acc_ref[0, 1, 1, 1]) == 9 * C * 255 * 255
+    xd, wd = _dev(x, cuda), _dev(w, cuda)
+    sa_d, sw_d = mpq.absmax(xd), mpq.absmax(wd, mpq.SCALE_PER_ROW)
+    xp = mpq.encode_nchw(xd, sa_d, 8)
+    wp, taps = mpq.encode_oihw(wd, sw_d, 8, mpq.SCALE_PER_ROW)
+    yi = torch.empty(acc_ref.shape, dtype=torch.int32, device=cuda)
+    yf = torch.empty(acc_ref.shape, dtype=torch.float32, device=cuda)
+    mpq.conv(xp, 8, 1, C, 4, 4, wp, 8, taps, O, 3, 3, 1, 1, yi, yf, sa_d, sw_d, mpq.SCALE_PER_ROW)
+    assert np.array_equal(yi.cpu().numpy(), acc_ref)
+    assert rel_close(yf.cpu().numpy(), out_ref)
+
+
 def test_conv_1x1_equals_gemm(mpq, cuda):
     """A 1x1 stride-1 convolution is the GEMM of the pixel matrix with the weight matrix."""
     x = inputs.uniform_levels(7, 1, (2, 128, 6, 5), 4)
