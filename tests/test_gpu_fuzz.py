@@ -82,3 +82,26 @@ def test_gemm_very_tall_and_very_wide(mpq, cuda):
         mpq.gemm(mpq.encode(xd, sa_d, 2), 2, mpq.encode(wd, sw_d, 3), 3, m, n, k, ci, cf, sa_d, sw_d)
         assert np.array_equal(ci.cpu().numpy(), acc_ref)
         assert rel_close(cf.cpu().numpy(), out_ref)
+
+
+def test_two_streams_run_independent_layers(mpq, cuda):
+    """The entry points keep no hidden state between calls: two different layers issued alternately on
+    two side streams (so that their kernels interleave on the device) give the oracle's results."""
+    cases = []
+    for t, (m, n, k, ab, wb) in enumerate(((300, 500, 2000, 2, 2), (257, 390, 1500, 4, 3))):
+        x = inputs.uniform_levels(23, 2 * t, (m, k), ab)
+        w = inputs.uniform_levels(23, 2 * t + 1, (n, k), wb)
+        acc_ref, out_ref, _, _ = oracle.linear(x, w, ab, wb, w_per_row=True)
+        cases.append(dict(x=_dev(x, cuda), w=_dev(w, cuda), ab=ab, wb=wb, acc=acc_ref, out=out_ref,
+                          oi=torch.empty((m, n), dtype=torch.int32, device=cuda),
+                          of=torch.empty((m, n), dtype=torch.float32, device=cuda),
+                          stream=torch.cuda.Stream()))
+    torch.cuda.synchronize()
+    for _ in range(6):
+        for c in cases:
+            with torch.cuda.stream(c["stream"]):
+                mpq.linear(c["x"], c["w"], c["ab"], c["wb"], mpq.ACT_HTANH, mpq.SCALE_PER_ROW, c["oi"], c["of"])
+    torch.cuda.synchronize()
+    for c in cases:
+        assert np.array_equal(c["oi"].cpu().numpy(), c["acc"])
+        assert rel_close(c["of"].cpu().numpy(), c["out"])
