@@ -115,3 +115,18 @@ def test_stack_full_size_sampled(mpq, cuda):
                     ref = max(np.float32(ref) + shortcut[b, o, oh, ow], np.float32(0))
                 assert abs(float(yf[b, o, oh, ow]) - float(ref)) <= 1e-5 * abs(float(ref)), (name, b, o, oh, ow)
         layer_in = net.block_out[blk]
+
+
+def test_stack_repeated_forwards_are_identical(mpq, cuda):
+    """Back-to-back forwards on one stream (ranges are re-zeroed and re-raised every time, kernels of
+    consecutive forwards overlap at their edges): outputs and ranges repeat bit for bit."""
+    batch, size = 8, 96
+    net = QuantResNet18Stack(inputs.config5_weights(), batch, size, 4, 4, cuda, fused=True)
+    x = torch.from_numpy(inputs.config5_input(batch, size)).to(cuda)
+    first = net.forward(x).clone()
+    scales = net.scales.clone()
+    for _ in range(20):
+        out = net.forward(x)
+    torch.cuda.synchronize()
+    assert torch.equal(out, first) and torch.equal(net.scales, scales)
+    assert float(scales.min()) > 0
