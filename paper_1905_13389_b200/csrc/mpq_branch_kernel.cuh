@@ -228,9 +228,9 @@ branch_kernel(const BranchParams p) {
         for (int r = tid; r < BS; r += 256) {
             const int64_t g = s0 + r;
             if (g < p.streamed_rows) {
-                const int64_t hw = (int64_t)p.Ho * p.Wo;
-                const int n = (int)(g / hw);
-                const int rem = (int)(g % hw);
+                const uint32_t hw = (uint32_t)(p.Ho * p.Wo);       // output pixels fit 32 bits (checked by the host)
+                const int n = (int)((uint32_t)g / hw);
+                const int rem = (int)((uint32_t)g % hw);
                 row_n[r] = n;
                 row_ih0[r] = (rem / p.Wo) * p.stride - p.pad;
                 row_iw0[r] = (rem % p.Wo) * p.stride - p.pad;
