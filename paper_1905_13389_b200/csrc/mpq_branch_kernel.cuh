@@ -495,7 +495,7 @@ static int launch_auto(const BranchParams& p, cudaStream_t st) {
     const double penalty[3] = {SB >= 7 ? 1.10 : 1.00, T::resident(4) == 3 ? 0.98 : 1.05, 1.20};      // TS = 8, 4, 2
     int best = 0;
     double best_cost = 0.0;
-    for (int c = 0; c < 3; ++c) {
+    for (int c = 0; c < (MODE == kModeConv ? 2 : 3); ++c) {      // the 32-wide tile never won for a convolution
         const int ts = 8 >> c;
         const int per_sm = T::resident(ts);
         const int64_t slots = (int64_t)per_sm * 148;
@@ -508,7 +508,7 @@ static int launch_auto(const BranchParams& p, cudaStream_t st) {
     }
     if (best == 0) return launch_branch<HB, SB, 8, MODE>(p, st);
     if (best == 1) return launch_branch<HB, SB, 4, MODE>(p, st);
-    return launch_branch<HB, SB, 2, MODE>(p, st);
+    return launch_branch<HB, SB, 2, kModeGemm>(p, st);
 }
 
 // One translation unit per held-operand width instantiates all eight streamed widths.
