@@ -47,6 +47,75 @@ def _peaks():
     return {"hbm_gbs": HBM_FALLBACK_GBS}, "fallback"
 
 
+class NvmlClockSampler:
+    """Reads SM clock, power and clock-event reasons through NVML every 5 ms in a thread while the timed
+    region runs (read-only queries; nothing on the GPU is set).  ``mark()`` brackets the timed region:
+    the summary uses the samples taken inside it."""
+    REASONS = (("hw_slowdown", "nvmlClocksEventReasonHwSlowdown"),
+               ("hw_thermal_slowdown", "nvmlClocksEventReasonHwThermalSlowdown"),
+               ("sw_thermal_slowdown", "nvmlClocksEventReasonSwThermalSlowdown"),
+               ("sw_power_cap", "nvmlClocksEventReasonSwPowerCap"))
+
+    def __init__(self, torch_index: int):
+        import pynvml
+        import torch
+        self.nv = pynvml
+        pynvml.nvmlInit()
+        props = torch.cuda.get_device_properties(torch_index)
+        try:
+            bus = "%08X:%02X:%02X.0" % (props.pci_domain_id, props.pci_bus_id, props.pci_device_id)
+            self.handle = pynvml.nvmlDeviceGetHandleByPciBusId(bus.encode())
+        except Exception:
+            self.handle = pynvml.nvmlDeviceGetHandleByIndex(torch_index)
+        self.samples = []                       # (time, sm_mhz, reasons bitmask)
+        self.max_mhz = float(pynvml.nvmlDeviceGetMaxClockInfo(self.handle, pynvml.NVML_CLOCK_SM))
+        self.marks = []
+        self.stop = threading.Event()
+        self.thread = threading.Thread(target=self._run, daemon=True)
+
+    def _run(self):
+        nv = self.nv
+        while not self.stop.is_set():
+            try:
+                mhz = float(nv.nvmlDeviceGetClockInfo(self.handle, nv.NVML_CLOCK_SM))
+                mask = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self.handle))
+                self.samples.append((time.perf_counter(), mhz, mask))
+            except Exception:
+                pass
+            time.sleep(0.005)
+
+    def __enter__(self):
+        self.thread.start()
+        return self
+
+    def mark(self):
+        self.marks.append(time.perf_counter())
+
+    def __exit__(self, *exc):
+        self.stop.set()
+        self.thread.join(timeout=2)
+
+    def summary(self):
+        lo, hi = (self.marks[0], self.marks[-1]) if len(self.marks) >= 2 else (0.0, float("inf"))
+        inside = [s for s in self.samples if lo <= s[0] <= hi] or self.samples
+        if not inside:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "samples": 0}
+        mask = 0
+        for s in inside:
+            mask |= s[2]
+        reasons = sorted(name for name, attr in self.REASONS if mask & int(getattr(self.nv, attr, 0)))
+        return {"sm_mhz": statistics.median(s[1] for s in inside), "sm_max_mhz": self.max_mhz, "reasons": reasons,
+                "samples": len(inside), "source": "NVML, 5 ms period, inside the timed region"}
+
+
+def clock_sampler(index: int):
+    """NVML sampler when the NVML binding is importable, else the nvidia-smi one."""
+    try:
+        return NvmlClockSampler(index)
+    except Exception:
+        return ClockSampler(index)
+
+
 class ClockSampler:
     """Samples nvidia-smi clocks and throttle reasons every 200 ms while the timed region runs."""
     QUERY = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
@@ -57,6 +126,9 @@ class ClockSampler:
         self.index = index
         self.rows = []
         self.proc = None
+
+    def mark(self):
+        pass
 
     def __enter__(self):
         try:
@@ -258,14 +330,16 @@ def run_cuda(args):
     mix_rate, _, _ = mpq.measure_mix_peak(4)                # 4 logic ops + 1 POPC + 1 multiply-add per group
     branch_peak = 2.0 * mix_rate                            # one group stands for two algorithmic word-popcounts
 
-    with ClockSampler(local_rank) as clocks:
+    with clock_sampler(local_rank) as clocks:
         barrier()
+        clocks.mark()
         t0, t1 = ev(), ev()
         t0.record()
         for _ in range(args.steps):
             step(True)
         t1.record()
         barrier()
+        clocks.mark()
     elapsed_ms = max_over_ranks(t0.elapsed_time(t1), world, dev)
     ms_per_step = elapsed_ms / args.steps
     value = whole_job_tops(world, m, n, k, ms_per_step)
