@@ -74,7 +74,7 @@ int mpq_absmax(const float* x, int64_t rows, int64_t k, int64_t ldx, int mode, i
                float* scale_out, void* stream);
 
 /* ---- Encoder (Fig. 1 "Encoder"; quantizer Eq. 15 with round-half-up; code Table 2 / Eq. 10;
- * one bit per element, Section 1 "store by bit vectors").
+ * one bit per element, the bit-vector storage of Section 1).
  * Per element, in fp32: inv = 1/s (0 if s is not a finite positive number),
  * y = (x*inv) * ((2^bits-1)/2) as two rounded multiplies, NaN -> 0, HReLU: max(y,0),
  * clamp to [-2^(bits-1), 2^(bits-1)-1/2], u = floor(y) + 2^(bits-1).  Plane p gets bit p of u.
@@ -103,13 +103,13 @@ int mpq_encode_oihw(const float* w, int O, int C, int KH, int KW, const float* s
  *   c_f32    = float(c_i32) * ((a_scale/(2^a_bits-1)) * (b_scale[c]/(2^b_bits-1)))
  * c_i32 and c_f32 are [m x n] row-major with row stride ldc; either may be NULL, not both.
  * a_scale: 1 value; b_scale: 1 value (PER_TENSOR) or n values (PER_ROW); both may be NULL
- * when c_f32 is NULL.  No bias ("we suppose the bias does not exist"). */
+ * when c_f32 is NULL.  No bias term (Section 3.1 sets it aside). */
 int mpq_gemm(const uint32_t* a_planes, int a_bits, const uint32_t* b_planes, int b_bits,
              int64_t m, int64_t n, int64_t k,
              int32_t* c_i32, float* c_f32, int64_t ldc,
              const float* a_scale, const float* b_scale, int b_mode, void* stream);
 
-/* ---- Convolution by the same decomposition ("convolution ... layers are also suit"),
+/* ---- Convolution by the same decomposition (Section 3.1 extends it to convolutions),
  * done as an implicit im2col on the packed planes: GEMM row = output pixel (n, oh, ow),
  * GEMM k = (kh, kw, c).  x_planes from mpq_encode_nchw, w_planes and tap_sums from
  * mpq_encode_oihw.  3x3 or 1x1, stride 1 or 2, pad 0 or 1, true zero padding (a tap outside

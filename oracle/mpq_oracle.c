@@ -106,13 +106,6 @@ int64_t mpq_oracle_gemm(const int16_t* qa, const int16_t* qb,
     return overflow;
 }
 
-/* Rows [r0, r1) only, all columns: used to sample a large problem. */
-int64_t mpq_oracle_gemm_rows(const int16_t* qa, const int16_t* qb,
-                             int64_t r0, int64_t r1, int64_t n, int64_t k, int32_t* acc_rows)
-{
-    return mpq_oracle_gemm(qa + r0 * k, qb, r1 - r0, n, k, acc_rows);
-}
-
 /* ---- a6: direct convolution on the decoded integers ----
  * qx [N][C][H][W], qw [O][C][KH][KW], acc [N][O][Ho][Wo],
  * Ho = (H + 2 pad - KH)/stride + 1.  Out-of-image taps add 0. */

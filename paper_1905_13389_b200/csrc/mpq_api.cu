@@ -112,7 +112,6 @@ extern "C" int mpq_linear(const float* x, const float* w, int64_t m, int64_t n, 
 static __device__ __align__(256) unsigned char g_linear_static_scratch[MPQ_LINEAR_STATIC_BYTES];
 
 namespace {
-constexpr int kMaxDevices = 64;
 std::mutex g_static_mutex;
 unsigned char* g_static_ptr[kMaxDevices] = {};   // device address of the scratch, per device
 

@@ -469,15 +469,8 @@ static int launch_branch(const BranchParams& p, cudaStream_t st) {
     constexpr int BH = 16 * T::TH, BS = 16 * TS;
     constexpr size_t smem_bytes = (size_t)T::STAGES * (HB * T::KQ * BH + SB * T::KQ * BS) * sizeof(uint4);
     auto kern = branch_kernel<HB, SB, TS, MODE>;
-    static bool configured = false;   // per instantiation; attribute is per function, set once per process+device
-    static int configured_dev = -1;
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return MPQ_ERR_CUDA;
-    if (!configured || configured_dev != dev) {
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes) != cudaSuccess)
-            return MPQ_ERR_CUDA;
-        configured = true; configured_dev = dev;
-    }
+    static PerDeviceOnce configured;   // per instantiation: the attribute belongs to (function, device)
+    if (configured.raise_smem_limit(kern, smem_bytes) != MPQ_OK) return MPQ_ERR_CUDA;
     const int64_t blocks = ceil_div(p.streamed_rows, BS) * ceil_div(p.held_rows, BH);
     if (blocks <= 0 || blocks > 0x7fffffffLL) return MPQ_ERR_BAD_SHAPE;
     return launch_chained(kern, (unsigned)blocks, 256, smem_bytes, st, p);
@@ -485,12 +478,14 @@ static int launch_branch(const BranchParams& p, cudaStream_t st) {
 
 // Streamed-side tile width (16*TS items): the widest tile has the least shared-memory traffic per
 // population count, but a grid of few large tiles leaves SMs idle in its last wave.  Pick the
-// width with the smallest estimated makespan: waves of (resident CTAs x 148 SMs) tiles, each
+// width with the smallest estimated makespan: waves of (resident CTAs x SM count) tiles, each
 // costing its width times the CTAs that share an SM times a measured per-width inefficiency.
 template <int HB, int SB, int MODE>
 static int launch_auto(const BranchParams& p, cudaStream_t st) {
     using T = BranchTile<HB, SB>;
     const int64_t held_tiles = ceil_div(p.held_rows, 16 * T::TH);
+    const int sms = sm_count();
+    if (sms <= 0) return MPQ_ERR_CUDA;
     // (with 7 or 8 streamed planes the 128-wide tile's loop body outgrows the instruction cache)
     const double penalty[3] = {SB >= 7 ? 1.10 : 1.00, T::resident(4) == 3 ? 0.98 : 1.05, 1.20};      // TS = 8, 4, 2
     int best = 0;
@@ -498,7 +493,7 @@ static int launch_auto(const BranchParams& p, cudaStream_t st) {
     for (int c = 0; c < (MODE == kModeConv ? 2 : 3); ++c) {      // the 32-wide tile never won for a convolution
         const int ts = 8 >> c;
         const int per_sm = T::resident(ts);
-        const int64_t slots = (int64_t)per_sm * 148;
+        const int64_t slots = (int64_t)per_sm * sms;
         const int64_t tiles = ceil_div(p.streamed_rows, 16 * ts) * held_tiles;
         // a grid that fits the resident slots takes one tile time; a longer one its share of waves
         // plus half a wave of tail; a tile's time grows with its width and with the CTAs sharing the SM

@@ -2,6 +2,7 @@
 #pragma once
 #include <cuda_runtime.h>
 #include <stdint.h>
+#include <atomic>
 #include "mpq.h"
 
 namespace mpq {
@@ -17,6 +18,49 @@ inline bool bits_ok(int b) { return b >= 1 && b <= kMaxBits; }
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 inline int launch_status() { return cudaGetLastError() == cudaSuccess ? MPQ_OK : MPQ_ERR_CUDA; }
+
+// ---- Per-device host state ------------------------------------------------------------------
+// The only things the library remembers between calls are facts about a device that never change
+// while the process lives: its multiprocessor count and "this kernel's shared-memory limit has
+// been raised on this device".  Both sit in tables indexed by device ordinal and are written with
+// atomics, so concurrent host threads and processes that alternate between devices are safe
+// (a lost race only repeats an idempotent query or attribute call).
+constexpr int kMaxDevices = 64;
+
+inline int current_device() {
+    int dev = -1;
+    return (cudaGetDevice(&dev) == cudaSuccess && dev >= 0 && dev < kMaxDevices) ? dev : -1;
+}
+
+// Multiprocessors of the current device (0 if it cannot be read).
+inline int sm_count() {
+    static std::atomic<int> cached[kMaxDevices];
+    const int dev = current_device();
+    if (dev < 0) return 0;
+    int n = cached[dev].load(std::memory_order_relaxed);
+    if (n == 0) {
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
+        cached[dev].store(n, std::memory_order_relaxed);
+    }
+    return n;
+}
+
+// One flag per device for one kernel: set once that kernel's dynamic shared-memory limit has been
+// raised there.  A kernel's launcher keeps one static instance.
+struct PerDeviceOnce {
+    std::atomic<bool> done[kMaxDevices];
+    template <typename Kernel>
+    int raise_smem_limit(Kernel kernel, size_t bytes) {
+        const int dev = current_device();
+        if (dev < 0) return MPQ_ERR_CUDA;
+        if (!done[dev].load(std::memory_order_acquire)) {
+            if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess)
+                return MPQ_ERR_CUDA;
+            done[dev].store(true, std::memory_order_release);
+        }
+        return MPQ_OK;
+    }
+};
 
 // Rows [row0, row0 + rows) of the layer product (mpq_gemm on a row block of A): lets a caller
 // overlap the copy-out of finished rows with the product of the next ones.

@@ -69,7 +69,8 @@ absmax_kernel(const float* __restrict__ x, int64_t k, int64_t ldx, int64_t chunk
 // the quantizer and the bit split run on the floating-point pipe, the integer ALU sees one min
 // per element, and the plane stores are coalesced 128-byte rows.  The kernel is then limited by
 // HBM, not by issue slots.  A lane that meets a NaN (HTanh) or a degenerate range rebuilds its
-// words with the plain quantizer.
+// words with the plain quantizer (so does every lane when 1/s overflows to infinity, which a
+// positive subnormal range does: a zero element then gives 0 * inf = NaN without being one).
 //
 // Ragged or unaligned segments take the ballot path: in step j lane L quantizes element
 // 32 j + L and one __ballot_sync per plane transposes that bit across the warp into word j.
@@ -133,7 +134,7 @@ encode_rows_kernel(const float* __restrict__ x, int64_t rows, int64_t k, int64_t
         uint32_t word[BITS];
 #pragma unroll
         for (int p = 0; p < BITS; ++p) word[p] = lw.word(p);
-        if (ACT == MPQ_ACT_HTANH && (probe != probe || inv == 0.0f)) {
+        if (ACT == MPQ_ACT_HTANH && (probe != probe || inv == 0.0f || inv == __int_as_float(0x7f800000))) {
 #pragma unroll
             for (int p = 0; p < BITS; ++p) word[p] = 0u;
             for (int t = 0; t < 32; ++t) {
@@ -224,7 +225,7 @@ encode_nchw_kernel(const float* __restrict__ x, int N, int C, int64_t HW,
     uint32_t word[BITS];
 #pragma unroll
     for (int p = 0; p < BITS; ++p) word[p] = lw.word(p);
-    if (ACT == MPQ_ACT_HTANH && (probe != probe || inv == 0.0f)) {
+    if (ACT == MPQ_ACT_HTANH && (probe != probe || inv == 0.0f || inv == __int_as_float(0x7f800000))) {
 #pragma unroll
         for (int p = 0; p < BITS; ++p) word[p] = 0u;
         for (int c = 0; c < 32; ++c) {
@@ -400,6 +401,8 @@ extern "C" int mpq_encode_oihw(const float* w, int O, int C, int KH, int KW, con
 extern "C" int mpq_add_relu(const float* a, const float* b, float* y, int64_t n, void* stream) {
     if (!a || !y) return MPQ_ERR_NULL;
     if (n <= 0) return MPQ_ERR_BAD_SHAPE;
-    const int64_t blocks = min((int64_t)148 * 16, ceil_div(n, 256));
+    const int sms = sm_count();
+    if (sms <= 0) return MPQ_ERR_CUDA;
+    const int64_t blocks = min((int64_t)sms * 16, ceil_div(n, 256));
     return launch_chained(add_relu_kernel, (unsigned)blocks, 256, 0, (cudaStream_t)stream, a, b, y, n);
 }

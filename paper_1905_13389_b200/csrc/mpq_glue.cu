@@ -159,14 +159,8 @@ extern "C" int mpq_stem_conv7x7(const float* x, const float* w, float* y, int N,
     const int64_t blocks = (int64_t)N * ceil_div(Ho, kStemRows) * ceil_div(Wo, kStemCols);
     if (blocks > 0x7fffffffLL) return MPQ_ERR_BAD_SHAPE;
     const size_t smem = (size_t)(kStemTaps * kStemWRow + 3 * kStemPatchH * kStemPatchStride) * sizeof(float);
-    static bool configured[64] = {};
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return MPQ_ERR_CUDA;
-    if (!configured[dev]) {
-        if (cudaFuncSetAttribute(stem_conv7x7_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-            return MPQ_ERR_CUDA;
-        configured[dev] = true;
-    }
+    static PerDeviceOnce configured;
+    if (configured.raise_smem_limit(stem_conv7x7_kernel, smem) != MPQ_OK) return MPQ_ERR_CUDA;
     return launch_chained(stem_conv7x7_kernel, (unsigned)blocks, kStemThreads, smem, (cudaStream_t)stream,
                           x, w, y, N, H, W, Ho, Wo, relu);
 }
@@ -177,7 +171,9 @@ extern "C" int mpq_maxpool3x3s2(const float* x, float* y, int N, int C, int H, i
     if (N <= 0 || C <= 0 || H <= 0 || W <= 0) return MPQ_ERR_BAD_SHAPE;
     const int Ho = (H + 2 - 3) / 2 + 1, Wo = (W + 2 - 3) / 2 + 1;
     const int64_t total = (int64_t)N * C * Ho * ((Wo + 3) / 4);
-    const int64_t blocks = min((int64_t)148 * 32, ceil_div(total, 256));
+    const int sms = sm_count();
+    if (sms <= 0) return MPQ_ERR_CUDA;
+    const int64_t blocks = min((int64_t)sms * 32, ceil_div(total, 256));
     return launch_chained(maxpool3x3s2_kernel, (unsigned)blocks, 256, 0, (cudaStream_t)stream,
                           x, y, (int64_t)N * C, H, W, Ho, Wo, out_max);
 }

@@ -12,6 +12,25 @@ def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: needs a CUDA device (run with -m gpu on a B200)")
 
 
+def pytest_collection_modifyitems(config, items):
+    """A plain `pytest tests/` on a machine without a CUDA device runs the CPU suite only: the
+    GPU-marked tests are deselected unless a marker expression (-m gpu) asked for them."""
+    if config.option.markexpr:
+        return
+    try:
+        import torch
+        have_gpu = torch.cuda.is_available()
+    except Exception:
+        have_gpu = False
+    if have_gpu:
+        return
+    keep = [it for it in items if "gpu" not in it.keywords]
+    dropped = [it for it in items if "gpu" in it.keywords]
+    if dropped:
+        config.hook.pytest_deselected(items=dropped)
+        items[:] = keep
+
+
 @pytest.fixture(scope="session")
 def golden_dir():
     return os.path.join(ROOT, "tests", "golden")

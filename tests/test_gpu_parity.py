@@ -91,6 +91,26 @@ def test_encode_degenerate_scale(mpq, cuda):
         assert u.tolist() == [[4] * 6]                    # q = +1 everywhere
 
 
+@pytest.mark.parametrize("act", [0, 1])
+def test_encode_subnormal_scale_with_zeros(mpq, cuda, act):
+    """A positive subnormal range makes 1/s overflow to infinity, so an exact zero gives 0 * inf = NaN
+    and must land on the level above zero on every path: full 1024-element rows (lane-local path),
+    a ragged row (ballot path) and the NCHW encoder."""
+    rng = np.random.default_rng(40)
+    s = np.array([1e-40], np.float32)
+    assert 0.0 < float(s[0]) < 2.9e-39
+    for shape in ((3, 1024), (2, 777)):
+        x = (rng.standard_normal(shape) * 1e-39).astype(np.float32)
+        x[:, ::5] = 0.0
+        u = unpack_planes(mpq.encode(_dev(x, cuda), _dev(s, cuda), 3, 0, act).cpu().numpy(), shape[1])
+        assert np.array_equal(u, oracle.levels(oracle.quantize(x, s, 3, act=act), 3))
+    xn = (rng.standard_normal((2, 32, 5, 7)) * 1e-39).astype(np.float32)
+    xn[:, ::3] = 0.0
+    planes = mpq.encode_nchw(_dev(xn, cuda), _dev(s, cuda), 3, act).cpu().numpy()      # [bits][N][H][W][1]
+    u = unpack_planes(planes.reshape(3, -1, 1), 32).reshape(2, 5, 7, 32).transpose(0, 3, 1, 2)
+    assert np.array_equal(u, oracle.levels(oracle.quantize(xn, s, 3, act=act), 3))
+
+
 @pytest.mark.parametrize("bits", [1, 2, 4, 7])
 def test_encode_rows_full_segments_with_specials(mpq, cuda, bits):
     """Full 1024-element segments (the lean path) holding NaN, +-inf, exact ties, values far

@@ -236,3 +236,58 @@ def test_layer_helpers_compose_the_steps():
     assert np.array_equal(acc, qa @ qb.T)
     ref = acc.astype(np.float64) * float(s_a[0]) * s_w.astype(np.float64)[None, :] / 9.0
     assert np.all(np.abs(out - ref) <= 1e-6 * np.abs(ref))
+
+
+@pytest.mark.parametrize("a_bits,w_bits", [(2, 2), (4, 3)])
+def test_scale_on_nchw_accumulators(a_bits, w_bits):
+    """The decoder scale on a convolution's [N][O][Ho][Wo] accumulators: the weight range of
+    output channel o multiplies every pixel of channel o and nothing else.  Checked element by
+    element against Eq. 18 in exact rationals, and against the 2-D path applied per channel."""
+    rng = np.random.default_rng(67)
+    N, O, Ho, Wo = 3, 5, 4, 6
+    acc = rng.integers(-2 ** 20, 2 ** 20, size=(N, O, Ho, Wo)).astype(np.int32)
+    s_a = np.float32(1.9)
+    s_w = rng.uniform(0.05, 3.0, size=O).astype(np.float32)     # all different: a wrong channel index shows
+    La, Lw = 2 ** a_bits - 1, 2 ** w_bits - 1
+    out32 = oracle.scale(acc, s_a, s_w, a_bits, w_bits)
+    out64 = oracle.scale_f64(acc, s_a, s_w, a_bits, w_bits)
+    assert out32.shape == acc.shape and out64.shape == acc.shape
+    for idx in np.ndindex(N, O, Ho, Wo):
+        exact = Fraction(int(acc[idx])) * Fraction(float(s_a)) * Fraction(float(s_w[idx[1]])) / (La * Lw)
+        assert abs(out64[idx] - float(exact)) <= 1e-14 * abs(float(exact))
+        assert abs(float(out32[idx]) - float(exact)) <= 4 * 2.0 ** -24 * abs(float(exact)) * 1.01
+    # the 2-D path (rows = pixels, columns = channels) gives the same bits
+    flat = acc.transpose(0, 2, 3, 1).reshape(-1, O)
+    ref2d = oracle.scale(flat, s_a, s_w, a_bits, w_bits).reshape(N, Ho, Wo, O).transpose(0, 3, 1, 2)
+    assert np.array_equal(out32, ref2d)
+    # one weight range for the whole tensor
+    one = oracle.scale(acc, s_a, s_w[2:3], a_bits, w_bits)
+    assert np.array_equal(one[:, 2], out32[:, 2])
+
+
+@pytest.mark.parametrize("per_channel", [True, False])
+@pytest.mark.parametrize("act", [oracle.HTANH, oracle.HRELU])
+def test_conv_layer_composes_the_steps(per_channel, act):
+    """The whole encoded convolution layer against its parts put together by hand: numpy ranges,
+    the (separately pinned) quantizer, a matmul on a materialised im2col, Eq. 18 in rationals."""
+    rng = np.random.default_rng(71 + int(per_channel) + 2 * act)
+    N, C, H, W, O, a_bits, w_bits, stride, pad = 2, 6, 7, 5, 4, 3, 2, 2, 1
+    x = rng.standard_normal((N, C, H, W)).astype(np.float32)
+    w = (rng.standard_normal((O, C, 3, 3)) * rng.uniform(0.1, 2.0, size=(O, 1, 1, 1))).astype(np.float32)
+    acc, out, s_a, s_w = oracle.conv_layer(x, w, a_bits, w_bits, stride, pad, per_channel, act)
+    ref_sa = np.nanmax(np.maximum(x, 0)) if act == oracle.HRELU else np.nanmax(np.abs(x))
+    ref_sw = np.abs(w).reshape(O, -1).max(axis=1) if per_channel else np.abs(w).max(keepdims=True).reshape(1)
+    assert s_a.shape == (1,) and s_a[0] == ref_sa
+    assert np.array_equal(s_w, ref_sw)
+    qx = oracle.quantize(x, ref_sa, a_bits, act=act).astype(np.int64)
+    qw = np.stack([oracle.quantize(w[o], ref_sw[o if per_channel else 0], w_bits) for o in range(O)]).astype(np.int64)
+    if act == oracle.HRELU:
+        assert qx.min() >= 1                                     # the negative side sits on the level above zero
+    cols, Ho, Wo = _im2col(qx, 3, 3, stride, pad)
+    ref = (cols @ qw.reshape(O, -1).T).reshape(N, Ho, Wo, O).transpose(0, 3, 1, 2)
+    assert np.array_equal(acc, ref)
+    La, Lw = 2 ** a_bits - 1, 2 ** w_bits - 1
+    for idx in np.ndindex(*acc.shape):
+        sw = ref_sw[idx[1] if per_channel else 0]
+        exact = Fraction(int(ref[idx])) * Fraction(float(ref_sa)) * Fraction(float(sw)) / (La * Lw)
+        assert abs(float(out[idx]) - float(exact)) <= 4 * 2.0 ** -24 * abs(float(exact)) * 1.01

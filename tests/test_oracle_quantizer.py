@@ -198,3 +198,33 @@ def test_absmax_matches_numpy():
     assert np.array_equal(oracle.absmax(x, per_row=True), np.nanmax(np.abs(x), axis=1))
     assert oracle.absmax(x, act=oracle.HRELU)[0] == np.nanmax(np.maximum(x, 0))
     assert oracle.absmax(-np.abs(x), act=oracle.HRELU)[0] == 0.0
+
+
+def _eq15_level_of(x: Fraction, bits: int) -> int:
+    """Odd integer of Eq. 15 (round half up) for a real x, with the HTanh clamp to [-1, 1] first."""
+    L = 2 ** bits - 1
+    x = max(Fraction(-1), min(Fraction(1), x))
+    u = math.floor(L * (x + 1) / 2 + Fraction(1, 2))
+    return 2 * min(u, L) - L
+
+
+@pytest.mark.parametrize("s", [0.37, 3.7])
+@pytest.mark.parametrize("bits", [1, 2, 3, 5, 8])
+def test_eq15_of_x_over_s_for_ranges_that_are_not_powers_of_two(s, bits):
+    """With a range s that is not a power of two the code is Eq. 15 of the real quotient x/s
+    (exact rationals of the float32 inputs), for every input that is not within a few fp32
+    roundings of a level boundary (there the two rounded multiplies may legitimately decide
+    either way)."""
+    rng = np.random.default_rng(61 + bits)
+    s32 = np.float32(s)
+    x = (rng.uniform(-1.3, 1.3, 6000) * s).astype(np.float32)
+    L = 2 ** bits - 1
+    q = oracle.quantize(x, s32, bits).tolist()
+    checked = 0
+    for xi, qi in zip(x.tolist(), q):
+        t = Fraction(xi) / Fraction(float(s32)) * L / 2          # level boundaries are the integers of t
+        if abs(t - round(t)) <= 8 * Fraction(2) ** -23 * max(1, abs(t)):
+            continue
+        assert qi == _eq15_level_of(Fraction(xi) / Fraction(float(s32)), bits), (xi, qi)
+        checked += 1
+    assert checked > 5900
