@@ -9,7 +9,9 @@ throughput target is quoted on).  With N > 1 every rank runs the same workload o
 (independent problems, no exchange step): weak scaling, replicas only.
 
 Prints ONE JSON line (rank 0).  ``--impl reference`` times the CPU oracle instead.
-``--full FILE`` additionally writes per-workload numbers (sweep, FC, conv, encoders) to FILE.
+After the timed region the other workloads (fully-connected layer, convolution, bit-width sweep,
+ResNet-18-shaped stack, encoders) are timed too and a compact ``suite`` object is added to the line;
+``--full FILE`` additionally writes all their figures to FILE.
 """
 from __future__ import annotations
 
@@ -33,9 +35,10 @@ SIZE = 4096
 A_BITS = W_BITS = 2
 HBM_FALLBACK_GBS = 6650.0      # used only when MEASURED_PEAKS.json is absent
 # DRAM bytes per launch of the GEMM kernel (dram__bytes_read.sum + dram__bytes_write.sum) from the
-# committed ncu capture of this command, profiles/branch_kernel_w2a2_gemm4096.md: 8.46 MB + 80.40 MB.
+# kept ncu capture of this command: 8.46 MB + 80.40 MB.
 # Set back to None whenever branch_kernel changes after that capture.
 GEMM_DRAM_TRAFFIC_BYTES = 88.9e6
+ORACLE_SAMPLE_ROWS = 1024      # activation rows of the bounded sample the CPU oracle is timed on
 
 
 def _peaks():
@@ -253,11 +256,10 @@ def run_reference(args):
     if rank != 0:
         return
     x, w = _workload_arrays()
-    rows = 1024
-    tops, dt, cores, sample = _time_oracle(x, w, rows, args.steps, min(args.warmup, 1))
+    tops, dt, cores, sample = _time_oracle(x, w, ORACLE_SAMPLE_ROWS, args.steps, args.warmup)
     line = {
         "impl": "reference", "metric": METRIC, "value": tops, "unit": UNIT, "n_gpus": args.gpus,
-        "steps": args.steps, "warmup": min(args.warmup, 1), "ms_per_step": dt * 1e3, "higher_is_better": True,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "int32", "data": "synthetic",
         "config": _config(),
         "cpu_baseline": {"value": tops, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
@@ -325,9 +327,28 @@ def run_cuda(args):
     for _ in range(max(args.warmup, 3)):
         step(False)
     barrier()
-    popc_peak, probe_mhz, sms = mpq.measure_popc_peak()     # plain POPC issue rate, measured live
-    mix_rate, _, _ = mpq.measure_mix_peak(4)                # 4 logic ops + 1 POPC + 1 multiply-add per group
-    branch_peak = 2.0 * mix_rate                            # one group stands for two algorithmic word-popcounts
+    # Roofline denominators, all measured live with register-only probes at the clocks of this run:
+    # the plain POPC issue rate; the legacy one-bit tensor instruction; and the two integer pipes'
+    # joint issue rate for groups of L logic ops + 1 POPC + 1 multiply-add, L = 0..8.  A carry-save
+    # reduction that spends f full adders per xor word executes 1 + 2f logic ops and 1 - f POPCs per
+    # word, i.e. L = (1 + 2f)/(1 - f) logic ops per POPC and (L + 2)/3 algorithmic word-popcounts per
+    # group; the ceiling of the XOR/POPC route is the best of those over L.
+    popc_peak, probe_mhz, sms = mpq.measure_popc_peak()
+    mix_table = []
+    for L in range(0, 9):
+        rate, mhz_l, _ = mpq.measure_mix_peak(L)
+        words = (L + 2) / 3.0 if L >= 1 else 0.0           # L = 0 has no xor: not a branch product
+        mix_table.append({"logic_per_popc": L, "groups_per_s": rate, "probe_sm_mhz": mhz_l,
+                          "clk_per_warp_group_per_subpartition": 32.0 * 4 * sms * mhz_l * 1e6 / rate,
+                          "word_popc_per_group": words, "word_popc_per_s": rate * words})
+    own_mix_peak = mix_table[4]["word_popc_per_s"]         # the shipped kernel: one adder per two xor words, L = 4
+    best_mix = max(mix_table, key=lambda r: r["word_popc_per_s"])
+    branch_peak = best_mix["word_popc_per_s"]
+    b1 = {}
+    for name, and_popc in (("xor_popc", False), ("and_popc", True)):
+        rate, mhz_b, _ = mpq.measure_b1_mma_peak(and_popc)
+        b1[name] = {"warp_mma_per_s": rate, "warp_mma_per_clk_per_sm": rate / (mhz_b * 1e6 * sms),
+                    "word_popc_per_s": rate * 1024.0}
 
     with clock_sampler(local_rank) as clocks:
         barrier()
@@ -393,18 +414,28 @@ def run_cuda(args):
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "int32", "data": "synthetic",
-            "config": dict(_config(), binary_tops=value * A_BITS * W_BITS),
+            "config": _config(), "binary_tops": value * A_BITS * W_BITS,
             "roofline": {"bound": "alu", "kernel": "branch_kernel<2,2,4,gemm> (XOR + carry-save + POPC GEMM, 64 x 64 tile, 3 CTAs per SM)",
                          "achieved": achieved / 1e9, "peak": branch_peak / 1e9, "unit": "Gpopc/s",
                          "frac": achieved / branch_peak, "traffic": GEMM_DRAM_TRAFFIC_BYTES,
-                         "peak_source": "measured live at %.0f MHz on %d SMs: issue rate of the carry-save instruction mix "
-                                        "(4 three-input logic ops + 1 POPC + 1 integer multiply-add per group, "
-                                        "mpq_measure_mix_peak) x 2 algorithmic word-popcounts per group"
-                                        % (probe_mhz, sms),
+                         "peak_source": "measured live at %.0f MHz on %d SMs: the best, over L = 1..8, of the two integer "
+                                        "pipes' joint issue rate for groups of L three-input logic ops + 1 POPC + 1 integer "
+                                        "multiply-add (mpq_measure_mix_peak) x the (L + 2)/3 algorithmic word-popcounts a "
+                                        "carry-save reduction gets out of such a group; best L = %d"
+                                        % (probe_mhz, sms, best_mix["logic_per_popc"]),
+                         "frac_of_own_mix": achieved / own_mix_peak,
+                         "own_mix": "L = 4 (one full adder per two xor words): %.1f Gpopc/s" % (own_mix_peak / 1e9),
+                         "mix_table": mix_table,
                          "plain_popc_pipe": {"peak": popc_peak / 1e9, "frac": achieved / popc_peak,
                                              "lanes_per_clk_per_sm": popc_peak / (probe_mhz * 1e6 * sms),
                                              "note": "one POPC per xor word (no carry-save) cannot exceed this; the "
                                                      "kernel issues half as many POPCs as algorithmic popcounts"},
+                         "b1_mma": {"xor_popc": dict(b1["xor_popc"], frac=achieved / b1["xor_popc"]["word_popc_per_s"]),
+                                    "and_popc": dict(b1["and_popc"], frac=achieved / b1["and_popc"]["word_popc_per_s"]),
+                                    "note": "legacy mma.sync.m16n8k256 b1 in a register-only loop with constant operands "
+                                            "(mpq_measure_b1_mma_peak); one warp instruction = 1024 word-popcounts; frac = "
+                                            "achieved / that ceiling (above 1: the instruction is slower than this kernel "
+                                            "even with no operand traffic, so no tensor variant ships)"},
                          "ms_per_launch": gemm_ms, "algorithmic_popc_per_launch": popcs,
                          "equivalent_tops_of_this_kernel": 2.0 * m * n * k / (gemm_ms * 1e-3) / 1e12},
             "encode": {"bound": "hbm", "achieved": enc_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
@@ -421,18 +452,21 @@ def run_cuda(args):
             "gpu_launches": 5 * args.steps,
             "clocks": clocks.summary(),
         }
-        if world == 1 and not args.no_cpu_baseline:
-            tops, dt, cores, sample = _time_oracle(x_np, w_np, 1024, 4, 1)
-            line["cpu_baseline"] = {"value": tops, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample,
-                                    "seconds_per_sample": dt}
-        print(json.dumps(line), flush=True)
-        if args.full and world == 1:
+        suite = None
+        if world == 1 and not args.no_suite:
+            # the other workloads (fully-connected layer, convolution, sweep, stack, encoders), timed after
+            # the step above; a compact copy rides in this line, --full FILE keeps everything
             import bench_suite
             del x, w, ap, wp, ci, cf, xh, wh, oi, of, ws
             torch.cuda.empty_cache()
-            bench_suite.run_suite(dev, peaks["hbm_gbs"], args.full)
-            with open(args.full) as fh:
-                suite = json.load(fh)
+            suite = bench_suite.run_suite(dev, peaks["hbm_gbs"], args.full)
+            line["suite"] = bench_suite.compact(suite)
+        if world == 1 and not args.no_cpu_baseline:
+            tops, dt, cores, sample = _time_oracle(x_np, w_np, ORACLE_SAMPLE_ROWS, args.steps, args.warmup)
+            line["cpu_baseline"] = {"value": tops, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample,
+                                    "seconds_per_sample": dt}
+        print(json.dumps(line), flush=True)
+        if args.full and suite is not None:
             if not args.no_cpu_baseline:
                 suite["cpu_oracle"] = _oracle_other_workloads()
                 with open(args.full, "w") as fh:
@@ -450,6 +484,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-suite", action="store_true", help="skip the other workloads (only the timed step)")
     ap.add_argument("--full", metavar="FILE", default=None,
                     help="also time every workload (sweep, FC, conv, stack, encoders) and write them to FILE as JSON")
     args = ap.parse_args()

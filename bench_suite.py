@@ -50,7 +50,8 @@ def _graph_ms(fn, iters=20, warmup=5):
     return e0.elapsed_time(e1) / iters
 
 
-def run_suite(dev: torch.device, hbm_gbs: float, path: str):
+def run_suite(dev: torch.device, hbm_gbs: float, path=None):
+    """Times every workload; returns the figures as a dict and, when `path` is given, writes them there as JSON."""
     up = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(dev)
     popc_peak, mhz, sms = mpq.measure_popc_peak()
     mix, _, _ = mpq.measure_mix_peak(4)
@@ -214,14 +215,40 @@ def run_suite(dev: torch.device, hbm_gbs: float, path: str):
     enc["nchw_128x64x56x56_b4"] = {"us": ms * 1e3, "gb_s": by / (ms * 1e-3) / 1e9,
                                    "frac_of_hbm": by / (ms * 1e-3) / 1e9 / hbm_gbs}
     out["encoders"] = enc
-    with open(path, "w") as fh:
-        json.dump(out, fh, indent=1)
+    if path:
+        with open(path, "w") as fh:
+            json.dump(out, fh, indent=1)
     return out
+
+
+def compact(d: dict) -> dict:
+    """The suite's headline figures, small enough to ride in the benchmark's one JSON line.
+    `frac` = algorithmic word-popcounts per second / the carry-save mix peak measured in the same run."""
+    r3 = lambda v: round(float(v), 3)
+    c = {"peaks": {"mix_peak_gpopc_s": r3(d["branch_peak_gpopc_s"]), "plain_popc_gpopc_s": r3(d["popc_peak_gpopc_s"]),
+                   "hbm_gbs": d["hbm_gbs"]},
+         "gemm_w2a2_64x64x512": {"us": r3(d["gemm_w2a2_64x64x512"]["us"])}}
+    for name in ("fc_w2a2_64x4096x9216", "conv3x3_w3a3_32x256x14x14"):
+        r = d[name]
+        c[name] = {"us": r3(r["ms"] * 1e3), "equivalent_tops": r3(r["equivalent_tops"]), "frac": r3(r["frac_of_branch_peak"])}
+    c["conv3x3_w3a3_32x256x14x14"]["encode_nchw_us"] = r3(d["conv3x3_w3a3_32x256x14x14"]["encode_nchw_us"])
+    c["gemm_sweep_4096"] = {k: {"ms": r3(r["ms"]), "equivalent_tops": r3(r["equivalent_tops"]), "frac": r3(r["frac_of_branch_peak"])}
+                            for k, r in d["gemm_sweep_4096"].items()}
+    s = d["resnet18_stack_w4a4_b128"]
+    c["resnet18_stack_w4a4_b128"] = {
+        "ms_per_step": r3(s["ms_per_step"]), "images_per_s": round(s["images_per_s"], 1),
+        "quantized_layers_ms": r3(s["quantized_layers_ms"]),
+        "layers": {n: ([r3(r["ms"]), r3(r["frac_of_branch_peak"])] if "frac_of_branch_peak" in r else [r3(r["ms"])])
+                   for n, r in s["layers"].items()},
+        "layers_key": "[ms] or [ms, frac of mix peak]"}
+    c["encoders"] = {n: {"us": r3(r["us"]), "gb_s": round(r["gb_s"], 1), "frac_of_hbm": r3(r["frac_of_hbm"])}
+                     for n, r in d["encoders"].items()}
+    return c
 
 
 def summary_markdown(d: dict) -> str:
     """The suite's figures as the tables committed under profiles/."""
-    L = ["# Suite: all workloads on one B200 (`python bench.py --steps 20 --warmup 5 --full gpurun_out/suite.json`)\n",
+    L = ["# Suite: all workloads on one B200 (`python bench.py --steps 20 --warmup 5 --full FILE`)\n",
          "CUDA events on the launching stream after warm-up; short kernels replayed from a CUDA graph (no host launch",
          "gaps).  Peaks measured in the same run: plain POPC pipe %.0f Gpopc/s, carry-save mix peak %.0f Gpopc/s"
          % (d["popc_peak_gpopc_s"], d["branch_peak_gpopc_s"]),

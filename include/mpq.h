@@ -218,6 +218,14 @@ int mpq_measure_popc_peak(double* popc_per_s, double* sm_mhz, int* sms, void* st
  * groups_per_s: lane-level groups per second over the whole chip. */
 int mpq_measure_mix_peak(int logic_per_popc, double* groups_per_s, double* sm_mhz, int* sms, void* stream);
 
+/* ---- Roofline denominator of the legacy one-bit tensor route for the binary branches (Eq. 7-10
+ * with the bitcount done by mma.sync.m16n8k256 on b1 operands): issue rate of that instruction in
+ * a register-only loop with constant operands, i.e. with no operand traffic at all.  and_popc = 0
+ * measures the xor.popc form (the branch product itself), 1 the and.popc form.  One warp-wide
+ * instruction stands for 16 * 8 * 256 / 32 = 1024 word-popcounts.  Synchronous.
+ * warp_mma_per_s: warp-level instructions per second over the whole chip. */
+int mpq_measure_b1_mma_peak(int and_popc, double* warp_mma_per_s, double* sm_mhz, int* sms, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

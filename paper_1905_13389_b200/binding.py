@@ -69,6 +69,9 @@ def lib() -> ctypes.CDLL:
         L.mpq_measure_mix_peak.argtypes = [i32, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double),
                                            ctypes.POINTER(ctypes.c_int), P]
         L.mpq_measure_mix_peak.restype = i32
+        L.mpq_measure_b1_mma_peak.argtypes = [i32, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double),
+                                              ctypes.POINTER(ctypes.c_int), P]
+        L.mpq_measure_b1_mma_peak.restype = i32
         for name in ("mpq_absmax", "mpq_encode", "mpq_encode_nchw", "mpq_encode_oihw", "mpq_gemm", "mpq_conv",
                      "mpq_add_relu", "mpq_stem_conv7x7", "mpq_maxpool3x3s2", "mpq_conv_fused", "mpq_zero", "mpq_linear", "mpq_linear_static", "mpq_linear_host", "mpq_measure_popc_peak"):
             getattr(L, name).restype = i32
@@ -309,4 +312,12 @@ def measure_mix_peak(logic_per_popc: int = 4):
     rate, mhz, sms = ctypes.c_double(), ctypes.c_double(), ctypes.c_int()
     _check(lib().mpq_measure_mix_peak(logic_per_popc, ctypes.byref(rate), ctypes.byref(mhz), ctypes.byref(sms),
                                       _stream()), "mpq_measure_mix_peak")
+    return rate.value, mhz.value, sms.value
+
+
+def measure_b1_mma_peak(and_popc: bool = False):
+    """(warp-level mma.sync.m16n8k256 b1 instructions per second over the chip, SM MHz, SM count)."""
+    rate, mhz, sms = ctypes.c_double(), ctypes.c_double(), ctypes.c_int()
+    _check(lib().mpq_measure_b1_mma_peak(int(and_popc), ctypes.byref(rate), ctypes.byref(mhz), ctypes.byref(sms),
+                                         _stream()), "mpq_measure_b1_mma_peak")
     return rate.value, mhz.value, sms.value

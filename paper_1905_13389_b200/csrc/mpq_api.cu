@@ -1,4 +1,4 @@
-// Status strings, size queries, the host-buffer fully-connected layer and the POPC-rate probe.
+// Status strings, size queries and the whole-layer entry points (device, built-in scratch, host buffers).
 #include <mutex>
 
 #include "mpq_common.cuh"
@@ -228,146 +228,4 @@ extern "C" int mpq_linear_host(const float* x_host, const float* w_host, int64_t
     if (cudaEventRecord(hp->copies_done, hp->copy_stream) != cudaSuccess) return MPQ_ERR_CUDA;
     if (cudaStreamWaitEvent(st, hp->copies_done, 0) != cudaSuccess) return MPQ_ERR_CUDA;
     return cudaStreamSynchronize(st) == cudaSuccess ? MPQ_OK : MPQ_ERR_CUDA;
-}
-
-// ---- POPC issue-rate probe ----------------------------------------------------------------
-namespace {
-constexpr int kProbeChains = 8;
-// The probe's few result words live in the module so that the call needs no buffer from the caller.
-__device__ unsigned long long probe_clk[2];
-__device__ uint32_t probe_sink[1];
-__global__ void popc_rate_kernel(uint32_t seed, int iters, uint32_t* sink, unsigned long long* clk) {
-    uint32_t x[kProbeChains];
-    const uint32_t s = seed ^ (threadIdx.x * 0x9E3779B9u);
-#pragma unroll
-    for (int i = 0; i < kProbeChains; ++i) x[i] = s * (uint32_t)(i + 3);
-    unsigned long long g0, g1;
-    const long long c0 = clock64();
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(g0));
-    for (int it = 0; it < iters; ++it) {
-#pragma unroll
-        for (int i = 0; i < kProbeChains; ++i) x[i] = __popc(x[i]) + s;   // independent chains
-    }
-    const long long c1 = clock64();
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(g1));
-    uint32_t r = 0;
-#pragma unroll
-    for (int i = 0; i < kProbeChains; ++i) r += x[i];
-    if (r == 0xFFFFFFFFu) sink[0] = r;          // never true: keeps the loop alive
-    if (threadIdx.x == 0 && blockIdx.x == 0) { clk[0] = (unsigned long long)(c1 - c0); clk[1] = g1 - g0; }
-}
-
-// The instruction mix of the carry-save branch kernel in a register-only loop: per group L
-// three-input logic operations, one population count and one integer multiply-add
-// (L = 4 when one full adder is spent per two xor words: per word 1 xor + 1 adder half-pair).
-template <int L>
-__global__ void mix_rate_kernel(uint32_t seed, uint32_t weight, int iters, uint32_t* sink, unsigned long long* clk) {
-    uint32_t a[kProbeChains], b[kProbeChains], c[kProbeChains];
-    const uint32_t s = seed ^ (threadIdx.x * 0x9E3779B9u);
-#pragma unroll
-    for (int i = 0; i < kProbeChains; ++i) { a[i] = s * (uint32_t)(i + 3); b[i] = ~a[i] * 7u; c[i] = 0u; }
-    unsigned long long g0, g1;
-    const long long c0 = clock64();
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(g0));
-    for (int it = 0; it < iters; ++it) {
-#pragma unroll
-        for (int i = 0; i < kProbeChains; ++i) {
-#pragma unroll
-            for (int l = 0; l < L; ++l) {
-                uint32_t d;
-                if (l & 1) asm("lop3.b32 %0, %1, %2, %3, 0xE8;" : "=r"(d) : "r"(a[i]), "r"(b[i]), "r"(s));
-                else       asm("lop3.b32 %0, %1, %2, %3, 0x96;" : "=r"(d) : "r"(a[i]), "r"(b[i]), "r"(s));
-                b[i] = a[i]; a[i] = d;
-            }
-            c[i] = (uint32_t)__popc(a[i]) * weight + c[i];
-            if (L == 0) a[i] = c[i];
-        }
-    }
-    const long long c1 = clock64();
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(g1));
-    uint32_t r = 0;
-#pragma unroll
-    for (int i = 0; i < kProbeChains; ++i) r += c[i] ^ a[i];
-    if (r == 0xFFFFFFFFu && weight == 0u) sink[0] = r;   // keeps the loop alive
-    if (threadIdx.x == 0 && blockIdx.x == 0) { clk[0] = (unsigned long long)(c1 - c0); clk[1] = g1 - g0; }
-}
-
-template <int L>
-void launch_mix(int blocks, int threads, uint32_t seed, int iters, uint32_t* sink, unsigned long long* clk, cudaStream_t st) {
-    mix_rate_kernel<L><<<blocks, threads, 0, st>>>(seed, 1u, iters, sink, clk);
-}
-}  // namespace
-
-extern "C" int mpq_measure_popc_peak(double* popc_per_s, double* sm_mhz, int* sms, void* stream) {
-    cudaStream_t st = (cudaStream_t)stream;
-    int dev = 0, n_sm = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return MPQ_ERR_CUDA;
-    if (cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return MPQ_ERR_CUDA;
-    unsigned long long* d_clk = nullptr; uint32_t* d_sink = nullptr;
-    if (cudaGetSymbolAddress((void**)&d_clk, probe_clk) != cudaSuccess) return MPQ_ERR_CUDA;
-    if (cudaGetSymbolAddress((void**)&d_sink, probe_sink) != cudaSuccess) return MPQ_ERR_CUDA;
-    const int threads = 512, blocks_per_sm = 2, iters = 20000;
-    cudaEvent_t e0, e1;
-    if (cudaEventCreate(&e0) != cudaSuccess || cudaEventCreate(&e1) != cudaSuccess) return MPQ_ERR_CUDA;
-    float best_ms = 1e30f; unsigned long long h_clk[2] = {0, 0}, best_clk[2] = {1, 1};
-    int rc = MPQ_OK;
-    for (int rep = 0; rep < 4 && rc == MPQ_OK; ++rep) {
-        cudaEventRecord(e0, st);
-        popc_rate_kernel<<<n_sm * blocks_per_sm, threads, 0, st>>>(12345u + rep, iters, d_sink, d_clk);
-        cudaEventRecord(e1, st);
-        if (cudaEventSynchronize(e1) != cudaSuccess || cudaGetLastError() != cudaSuccess) { rc = MPQ_ERR_CUDA; break; }
-        float ms = 0; cudaEventElapsedTime(&ms, e0, e1);
-        if (cudaMemcpy(h_clk, d_clk, sizeof(h_clk), cudaMemcpyDeviceToHost) != cudaSuccess) { rc = MPQ_ERR_CUDA; break; }
-        if (rep > 0 && ms < best_ms) { best_ms = ms; best_clk[0] = h_clk[0]; best_clk[1] = h_clk[1]; }
-    }
-    cudaEventDestroy(e0); cudaEventDestroy(e1);
-    if (rc != MPQ_OK) return rc;
-    const double popcs = (double)n_sm * blocks_per_sm * threads * (double)iters * kProbeChains;
-    if (popc_per_s) *popc_per_s = popcs / (best_ms * 1e-3);
-    if (sm_mhz) *sm_mhz = (double)best_clk[0] / (double)best_clk[1] * 1e3;
-    if (sms) *sms = n_sm;
-    return MPQ_OK;
-}
-
-extern "C" int mpq_measure_mix_peak(int logic_per_popc, double* groups_per_s, double* sm_mhz, int* sms, void* stream) {
-    if (logic_per_popc < 0 || logic_per_popc > 8) return MPQ_ERR_UNSUPPORTED;
-    cudaStream_t st = (cudaStream_t)stream;
-    int dev = 0, n_sm = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return MPQ_ERR_CUDA;
-    if (cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return MPQ_ERR_CUDA;
-    unsigned long long* d_clk = nullptr; uint32_t* d_sink = nullptr;
-    if (cudaGetSymbolAddress((void**)&d_clk, probe_clk) != cudaSuccess) return MPQ_ERR_CUDA;
-    if (cudaGetSymbolAddress((void**)&d_sink, probe_sink) != cudaSuccess) return MPQ_ERR_CUDA;
-    const int threads = 512, blocks_per_sm = 2, iters = 8000;
-    cudaEvent_t e0, e1;
-    if (cudaEventCreate(&e0) != cudaSuccess || cudaEventCreate(&e1) != cudaSuccess) return MPQ_ERR_CUDA;
-    float best_ms = 1e30f; unsigned long long h_clk[2] = {0, 0}, best_clk[2] = {1, 1};
-    int rc = MPQ_OK;
-    for (int rep = 0; rep < 4 && rc == MPQ_OK; ++rep) {
-        cudaEventRecord(e0, st);
-        const int blocks = n_sm * blocks_per_sm;
-        switch (logic_per_popc) {
-            case 0: launch_mix<0>(blocks, threads, 99u + rep, iters, d_sink, d_clk, st); break;
-            case 1: launch_mix<1>(blocks, threads, 99u + rep, iters, d_sink, d_clk, st); break;
-            case 2: launch_mix<2>(blocks, threads, 99u + rep, iters, d_sink, d_clk, st); break;
-            case 3: launch_mix<3>(blocks, threads, 99u + rep, iters, d_sink, d_clk, st); break;
-            case 4: launch_mix<4>(blocks, threads, 99u + rep, iters, d_sink, d_clk, st); break;
-            case 5: launch_mix<5>(blocks, threads, 99u + rep, iters, d_sink, d_clk, st); break;
-            case 6: launch_mix<6>(blocks, threads, 99u + rep, iters, d_sink, d_clk, st); break;
-            case 7: launch_mix<7>(blocks, threads, 99u + rep, iters, d_sink, d_clk, st); break;
-            default: launch_mix<8>(blocks, threads, 99u + rep, iters, d_sink, d_clk, st); break;
-        }
-        cudaEventRecord(e1, st);
-        if (cudaEventSynchronize(e1) != cudaSuccess || cudaGetLastError() != cudaSuccess) { rc = MPQ_ERR_CUDA; break; }
-        float ms = 0; cudaEventElapsedTime(&ms, e0, e1);
-        if (cudaMemcpy(h_clk, d_clk, sizeof(h_clk), cudaMemcpyDeviceToHost) != cudaSuccess) { rc = MPQ_ERR_CUDA; break; }
-        if (rep > 0 && ms < best_ms) { best_ms = ms; best_clk[0] = h_clk[0]; best_clk[1] = h_clk[1]; }
-    }
-    cudaEventDestroy(e0); cudaEventDestroy(e1);
-    if (rc != MPQ_OK) return rc;
-    const double groups = (double)n_sm * blocks_per_sm * threads * (double)iters * kProbeChains;
-    if (groups_per_s) *groups_per_s = groups / (best_ms * 1e-3);
-    if (sm_mhz) *sm_mhz = (double)best_clk[0] / (double)best_clk[1] * 1e3;
-    if (sms) *sms = n_sm;
-    return MPQ_OK;
 }

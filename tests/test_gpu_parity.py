@@ -536,3 +536,23 @@ def test_popc_peak_probe(mpq, cuda):
     assert sms >= 100 and 500 < mhz < 3000
     per_clk_sm = rate / (mhz * 1e6 * sms)
     assert 8 <= per_clk_sm <= 130          # lanes per clock per SM: a plausible pipe width
+
+
+def test_pipe_probes_are_sane(mpq, cuda):
+    """The roofline probes return rates in the range the SM's unit counts allow: the instruction mix
+    can only be slower than the plain population count, and the one-bit tensor instruction reports
+    a positive, finite rate."""
+    popc, mhz, sms = mpq.measure_popc_peak()
+    assert sms > 0 and 500 < mhz < 3000
+    lanes = popc / (mhz * 1e6 * sms)
+    assert 8 < lanes < 40                                    # POPC results per clock per SM
+    prev = None
+    for L in (0, 4, 8):
+        rate, _, _ = mpq.measure_mix_peak(L)
+        assert 0 < rate <= popc * 1.05
+        assert prev is None or rate <= prev * 1.05           # more logic per group never issues faster
+        prev = rate
+    for and_popc in (False, True):
+        rate, mhz_b, _ = mpq.measure_b1_mma_peak(and_popc)
+        per_clk = rate / (mhz_b * 1e6 * sms)
+        assert 0 < per_clk < 8                               # warp instructions per clock per SM
