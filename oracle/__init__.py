@@ -47,6 +47,8 @@ def _load():
             lib.mpq_oracle_absmax.restype = None
             lib.mpq_oracle_quantize.argtypes = [P, i64, i64, i64, P, i32, i32, i32, P]
             lib.mpq_oracle_quantize.restype = None
+            lib.mpq_oracle_quantize_trig.argtypes = [P, i64, i64, i64, P, i32, i32, i32, P]
+            lib.mpq_oracle_quantize_trig.restype = None
             lib.mpq_oracle_gemm.argtypes = [P, P, i64, i64, i64, P]
             lib.mpq_oracle_gemm.restype = i64
             lib.mpq_oracle_conv.argtypes = [P, i64, i64, i64, i64, P, i64, i64, i64, i64, i64, P]
@@ -106,6 +108,22 @@ def quantize(x, scale, bits: int, per_row: bool = False, act: int = HTANH) -> np
         raise ValueError("scale has %d entries, expected %d" % (scale.size, rows))
     q = np.empty(x.shape, dtype=np.int16)
     _load().mpq_oracle_quantize(_p(x), rows, k, k, _p(scale), int(per_row), bits, int(act), _p(q))
+    return q
+
+
+def quantize_trig(x, scale, bits: int, per_row: bool = False, act: int = HTANH) -> np.ndarray:
+    """The same codes through the trigonometric encoders (Eq. 11 and its family): each bit is the
+    sign of a sine of x/s.  Equal to :func:`quantize` except within a rounding of a level boundary."""
+    if not 1 <= bits <= 8:
+        raise ValueError("bits must be in 1..8")
+    x = _f32c(x)
+    scale = _f32c(np.atleast_1d(scale))
+    rows = x.shape[0] if per_row else 1
+    k = x.size // rows if rows else 0
+    if scale.size != rows:
+        raise ValueError("scale has %d entries, expected %d" % (scale.size, rows))
+    q = np.empty(x.shape, dtype=np.int16)
+    _load().mpq_oracle_quantize_trig(_p(x), rows, k, k, _p(scale), int(per_row), bits, int(act), _p(q))
     return q
 
 
@@ -184,6 +202,21 @@ def scale_f64(acc, s_a: float, s_w, a_bits: int, w_bits: int) -> np.ndarray:
     _load().mpq_oracle_scale_f64(_p(acc), outer, channels, inner, float(np.float32(s_a)), _p(s_w),
                                  int(per_channel), a_bits, w_bits, _p(out))
     return out
+
+
+def epilogue(out, bias=None, residual=None, relu: bool = False) -> np.ndarray:
+    """Glue after the decoder of a chained layer (not part of the paper's method, which has no bias):
+    out + bias[c] (one rounded fp32 add), + residual (one rounded fp32 add), then max(., 0).
+    ``out`` is [m][n] (bias per column) or [N][O][Ho][Wo] (bias per channel)."""
+    f = np.array(out, dtype=np.float32, copy=True)
+    if bias is not None:
+        b = _f32c(bias)
+        f = (f + (b[None, :] if f.ndim == 2 else b[None, :, None, None])).astype(np.float32)
+    if residual is not None:
+        f = (f + _f32c(residual)).astype(np.float32)
+    if relu:
+        f = np.where(f > 0, f, np.float32(0)).astype(np.float32)
+    return f
 
 
 def linear(x, w, a_bits: int, w_bits: int, w_per_row: bool = False, a_act: int = HTANH):

@@ -87,6 +87,50 @@ void mpq_oracle_quantize(const float* x, int64_t rows, int64_t k, int64_t ldx,
     }
 }
 
+/* ---- The encoder in its trigonometric form (Section 3.2, Eq. 11; other widths follow the same
+ * family: the highest bit has half a period on [-1,1] scaled by (2^b-1)/2^b, every lower bit
+ * doubles the frequency and flips the sign).  For y = clamp(x/s) in [-1,1]:
+ *     bit b-1 (highest)   = sign( sin((2^b-1)/2^b * pi * y))
+ *     bit m-1, 1 <= m < b = sign(-sin((2^b-1)/2^m * pi * y))
+ * with +1 stored as 1 and -1 as 0; the level index is the number those bits spell.
+ * At a zero of a sine (a level boundary, where Eq. 15 has a tie) the sign is that of the sine just
+ * ABOVE the zero, i.e. the sign of its slope there: the tie goes to the upper level, as the
+ * round-half-up reading of Eq. 15 does.  (x = 0 is a zero of every one of the sines; taking
+ * sign(0) = +1 for all of them would spell the top level.)
+ * The argument t = (2^b-1)/2^m * y is formed in fp32 (one rounded multiply: the multiplier is
+ * exact), the sine itself in double; a t that is a whole number is a zero of the sine.  This
+ * route and the level-index route (level_index above) agree except within a rounding of a zero
+ * of a sine, where each takes its own decision. */
+static int trig_level_index(float x, float inv_s, int bits, int hrelu)
+{
+    float y = x * inv_s;
+    if (y != y) y = 0.0f;                       /* NaN -> 0, the tie that goes to the level above zero */
+    if (hrelu && y < 0.0f) y = 0.0f;
+    if (y < -1.0f) y = -1.0f;
+    if (y > 1.0f) y = 1.0f;
+    const int L = (1 << bits) - 1;
+    int u = 0;
+    for (int m = 1; m <= bits; ++m) {
+        const float t = y * ((float)L / (float)(1 << m));
+        const double pi_t = 3.14159265358979323846 * (double)t;
+        double sine = (t == floorf(t)) ? cos(pi_t) : sin(pi_t);   /* at a zero: the slope's sign */
+        if (m < bits) sine = -sine;
+        if (sine > 0.0) u |= 1 << (m - 1);
+    }
+    return u;
+}
+
+void mpq_oracle_quantize_trig(const float* x, int64_t rows, int64_t k, int64_t ldx,
+                              const float* scale, int per_row, int bits, int hrelu, int16_t* q)
+{
+    const int L = (1 << bits) - 1;
+    for (int64_t r = 0; r < rows; ++r) {
+        const float inv = inverse_scale(per_row ? scale[r] : scale[0]);
+        for (int64_t t = 0; t < k; ++t)
+            q[r * k + t] = (int16_t)(2 * trig_level_index(x[r * ldx + t], inv, bits, hrelu) - L);
+    }
+}
+
 /* ---- a3+a4: acc[r][c] = sum_t qa[r][t] qb[c][t]   (Eq. 1-2) ----
  * Returns the number of outputs that do not fit int32 (0 when all fit). */
 int64_t mpq_oracle_gemm(const int16_t* qa, const int16_t* qb,

@@ -291,3 +291,22 @@ def test_conv_layer_composes_the_steps(per_channel, act):
         sw = ref_sw[idx[1] if per_channel else 0]
         exact = Fraction(int(ref[idx])) * Fraction(float(ref_sa)) * Fraction(float(sw)) / (La * Lw)
         assert abs(float(out[idx]) - float(exact)) <= 4 * 2.0 ** -24 * abs(float(exact)) * 1.01
+
+
+def test_epilogue_is_one_rounded_add_each():
+    """Bias, residual and max(., 0) after the decoder: each add rounds once in fp32, in that order."""
+    out = np.array([[1.0, -2.0, 3.0], [0.5, 16777216.0, -1.0]], dtype=np.float32)
+    bias = np.array([0.25, 1.0, -4.0], dtype=np.float32)
+    res = np.array([[1.0, 1.0, 1.0], [-1.0, 1.0, 0.5]], dtype=np.float32)
+    got = oracle.epilogue(out, bias, res, relu=True)
+    # 16777216 + 1 rounds back to 16777216 (tie to even), then + 1 does so again: two roundings, not one exact sum
+    assert got.tolist() == [[2.25, 0.0, 0.0], [0.0, 16777216.0, 0.0]]
+    assert oracle.epilogue(out, None, None, False).tolist() == out.tolist()
+    assert oracle.epilogue(out, bias).tolist() == [[1.25, -1.0, -1.0], [0.75, 16777216.0, -5.0]]
+    nchw = np.zeros((1, 3, 2, 2), dtype=np.float32)
+    assert oracle.epilogue(nchw, bias)[0, :, 1, 1].tolist() == bias.tolist()
+    rng = np.random.default_rng(89)
+    a, b, r = (rng.standard_normal((5, 7)).astype(np.float32) for _ in range(3))
+    ref = np.maximum(np.float32(1) * ((a.astype(np.float64) + b[0].astype(np.float64)).astype(np.float32).astype(np.float64)
+                                      + r.astype(np.float64)).astype(np.float32), 0)
+    assert np.array_equal(oracle.epilogue(a, b[0], r, True), ref)

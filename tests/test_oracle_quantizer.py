@@ -228,3 +228,49 @@ def test_eq15_of_x_over_s_for_ranges_that_are_not_powers_of_two(s, bits):
         assert qi == _eq15_level_of(Fraction(xi) / Fraction(float(s32)), bits), (xi, qi)
         checked += 1
     assert checked > 5900
+
+
+def test_trig_encoder_reproduces_table2(golden_dir):
+    """The trigonometric form (Eq. 11) sends Table 2's four printed levels to their printed states."""
+    rows = _read_table2(golden_dir)
+    x = np.array([float(fr) for fr, _, _ in rows], dtype=np.float32)
+    u = oracle.levels(oracle.quantize_trig(x, 1.0, 2), 2)
+    for (fr, hi, lo), ui in zip(rows, u.tolist()):
+        assert ((ui >> 1) & 1) * 2 - 1 == hi and (ui & 1) * 2 - 1 == lo
+
+
+@pytest.mark.parametrize("bits", range(1, 9))
+@pytest.mark.parametrize("act", [oracle.HTANH, oracle.HRELU])
+def test_trig_encoder_equals_eq15_away_from_level_boundaries(bits, act):
+    """Bit by bit the sine encoders spell the level index of Eq. 15 (exact rationals, round half up)
+    for every input that is not within a few roundings of a level boundary; at x = 0, a zero of every
+    sine, each sign is that of the sine just above the zero, which spells the level above zero (the
+    round-half-up tie); beyond the range the code saturates."""
+    rng = np.random.default_rng(83 + bits)
+    s32 = np.float32(1.7)
+    x = (rng.uniform(-1.4, 1.4, 5000) * 1.7).astype(np.float32)
+    x[:3] = [0.0, 40.0, -40.0]
+    L = 2 ** bits - 1
+    q = oracle.quantize_trig(x, s32, bits, act=act).tolist()
+    checked = 0
+    for xi, qi in zip(x.tolist(), q):
+        y = Fraction(xi) / Fraction(float(s32))
+        if act == oracle.HRELU:
+            y = max(y, Fraction(0))
+        t = y * L / 2
+        if y != 0 and abs(t) < 2 ** (bits - 1) and abs(t - round(t)) <= 8 * Fraction(2) ** -23 * max(1, abs(t)):
+            continue                                    # y == 0 is kept: the tie itself is pinned
+        assert qi == _eq15_level_of(y, bits), (xi, qi)
+        checked += 1
+    assert checked > 4900
+    assert q[0] == 1 and q[1] == L and q[2] == (1 if act == oracle.HRELU else -L)
+
+
+def test_trig_encoder_special_values():
+    """NaN takes the tie's level; an unusable range makes every code the level above zero."""
+    x = np.array([np.nan, -0.9, 0.9], np.float32)
+    assert oracle.quantize_trig(x, 1.0, 3).tolist() == [1, -7, 7]
+    for s in (0.0, -2.0, np.inf, np.nan):
+        assert oracle.quantize_trig(x, s, 3).tolist() == [1, 1, 1]
+    big = np.array([np.inf, -np.inf, 3e38], np.float32)
+    assert oracle.quantize_trig(big, 1.0, 2).tolist() == [3, -3, 3]
