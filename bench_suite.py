@@ -200,6 +200,12 @@ def run_suite(dev: torch.device, hbm_gbs: float, path=None):
         layers[name] = rec
     out["resnet18_stack_w4a4_b128"] = {"ms_per_step": ms, "images_per_s": batch / (ms * 1e-3),
                                        "quantized_layers_ms": quant_ms, "layers": layers}
+    # the same stack with ranges fixed beforehand (calibrated on this batch): every convolution writes its
+    # consumer's packed planes from its store, no encode pass after the first
+    static = QuantResNet18Stack(inputs.config5_weights(), batch, 224, 4, 4, dev, static_ranges=net.calibrated_ranges())
+    ms_static = _events_ms(lambda: static.forward(x), 5, 3)
+    out["resnet18_stack_w4a4_b128"]["static_ranges"] = {"ms_per_step": ms_static, "images_per_s": batch / (ms_static * 1e-3)}
+    del static
     # activation encoder of the first stage (NCHW variant, 102.8 MB in)
     xin = net.pooled
     i = [0]
@@ -238,6 +244,7 @@ def compact(d: dict) -> dict:
     c["resnet18_stack_w4a4_b128"] = {
         "ms_per_step": r3(s["ms_per_step"]), "images_per_s": round(s["images_per_s"], 1),
         "quantized_layers_ms": r3(s["quantized_layers_ms"]),
+        "static_ranges_ms_per_step": r3(s["static_ranges"]["ms_per_step"]),
         "layers": {n: ([r3(r["ms"]), r3(r["frac_of_branch_peak"])] if "frac_of_branch_peak" in r else [r3(r["ms"])])
                    for n, r in s["layers"].items()},
         "layers_key": "[ms] or [ms, frac of mix peak]"}
@@ -278,7 +285,9 @@ def summary_markdown(d: dict) -> str:
           % (s["ms_per_step"], s["images_per_s"]),
           "max(.,0) and every encoder's range ride in the producers' stores); encoded layers %.2f ms.  Span of an encoded"
           % s["quantized_layers_ms"],
-          "layer = encode_nchw + conv (shortcut convolutions reuse conv1's planes).\n",
+          "layer = encode_nchw + conv (shortcut convolutions reuse conv1's planes).  With ranges fixed beforehand",
+          "(every convolution writes its consumer's planes from its store): %.2f ms per step = %.0f images/s.\n"
+          % (s["static_ranges"]["ms_per_step"], s["static_ranges"]["images_per_s"]),
           "| layer | ms | frac of mix peak | frac of plain POPC pipe |", "|---|---|---|---|"]
     for n, r in s["layers"].items():
         if "frac_of_branch_peak" in r:
@@ -302,6 +311,7 @@ def _single(argv):
     """One product on its own, a few launches, for profiler captures:
         python bench_suite.py gemm A_BITS W_BITS SIZE
         python bench_suite.py conv BITS N C HW O KSIZE STRIDE
+        python bench_suite.py fc A_BITS W_BITS M N K
     Prints the CUDA-event time of the last 10 launches."""
     dev = torch.device("cuda:0")
     torch.cuda.set_device(0)
@@ -327,6 +337,15 @@ def _single(argv):
         fn = lambda: mpq.conv(xp, bits, N, C, HW, HW, wp, bits, taps, O, ks, ks, stride, pad, None, y, sa, sw,
                               mpq.SCALE_PER_ROW)
         popcs = float(bits * bits) * N * Ho * Ho * O * (ks * ks * C // 32)
+    elif argv[0] == "fc":
+        ab, wb, m, n, k = (int(a) for a in argv[1:6])
+        x = torch.randn(m, k, device=dev).relu_()
+        w = torch.randn(n, k, device=dev)
+        sa, sw = mpq.absmax(x, 0, mpq.ACT_HRELU), mpq.absmax(w, mpq.SCALE_PER_ROW)
+        ap, wp = mpq.encode(x, sa, ab, 0, mpq.ACT_HRELU), mpq.encode(w, sw, wb, mpq.SCALE_PER_ROW)
+        cf = torch.empty((m, n), dtype=torch.float32, device=dev)
+        fn = lambda: mpq.gemm(ap, ab, wp, wb, m, n, k, None, cf, sa, sw, mpq.SCALE_PER_ROW)
+        popcs = float(ab * wb) * m * n * (k // 32)
     else:
         raise SystemExit(_single.__doc__)
     ms = _events_ms(fn, 10, 4)

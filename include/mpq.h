@@ -13,8 +13,10 @@
  *   - Pointers are DEVICE pointers unless the name ends in _host.  The caller owns and
  *     sizes every buffer; the library allocates no device memory and keeps no state between
  *     calls (mpq_linear and mpq_linear_host stage through a caller-provided device workspace).
- *     Two documented exceptions: mpq_linear_static works on a buffer built into the library
- *     image, and mpq_linear_host keeps one helper stream and a few events per device.
+ *     Documented exceptions: mpq_linear_static works on a buffer built into the library image;
+ *     mpq_linear_host / mpq_linear_host_prepared keep one helper stream and a few events per
+ *     device; and per device the library remembers the multiprocessor count and which kernels
+ *     have had their shared-memory limit raised (facts that never change while the process lives).
  *   - Calls are asynchronous on `stream` (a cudaStream_t passed as void*; NULL = the
  *     default stream) unless stated otherwise.  Outputs are fully overwritten.
  *   - Return value: an mpq_status.  Errors that the host can see (null pointers, bad
@@ -58,6 +60,10 @@ typedef enum { MPQ_SCALE_PER_TENSOR = 0, MPQ_SCALE_PER_ROW = 1 } mpq_scale_mode;
  * HReLU clamps it to [0,1] (negative inputs land on the level just above zero). */
 typedef enum { MPQ_ACT_HTANH = 0, MPQ_ACT_HRELU = 1 } mpq_act;
 
+/* Form of the Encoder: the level-index route (quantizer of Eq. 15, the fast path) or the
+ * trigonometric encoders of Section 3.2 (Eq. 11 and its family), one sine per bit. */
+typedef enum { MPQ_ENC_LEVELS = 0, MPQ_ENC_TRIG = 1 } mpq_encoder;
+
 const char* mpq_status_string(int status);
 
 /* Words per packed row: ceil(k/32) rounded up to a multiple of 4 (rows are 16-byte multiples).
@@ -82,6 +88,21 @@ int mpq_absmax(const float* x, int64_t rows, int64_t k, int64_t ldx, int mode, i
 int mpq_encode(const float* x, int64_t rows, int64_t k, int64_t ldx,
                const float* scale, int mode, int act, int bits,
                uint32_t* planes, void* stream);
+
+/* The same call with the form of the Encoder selectable (Section 3.2 "M-bit Encoding Functions").
+ * MPQ_ENC_LEVELS is mpq_encode.  MPQ_ENC_TRIG evaluates the paper's periodic encoders literally:
+ * with y = x/s limited by `act` to [-1,1] (HTanh) or [0,1] (HReLU) and L = 2^bits - 1,
+ *     bit bits-1 (highest)   = sign( sin(L/2^bits * pi * y)),
+ *     bit m-1, 1 <= m < bits = sign(-sin(L/2^m * pi * y))
+ * (Eq. 11 is the case bits = 2; other widths continue the family: the highest bit has half a period
+ * on [-1,1], each lower bit doubles the frequency).  Each argument L/2^m * y is one rounded fp32
+ * multiply.  At a zero of a sine -- a level boundary, a tie of Eq. 15 -- the sign is that of the
+ * sine just above the zero, so ties go to the upper level as in mpq_encode and x = 0 lands on the
+ * level above zero.  The two forms give the same planes except for inputs within one fp32 rounding
+ * of a level boundary, where each takes its own decision.  A reference form, not tuned. */
+int mpq_encode_with(int encoder, const float* x, int64_t rows, int64_t k, int64_t ldx,
+                    const float* scale, int mode, int act, int bits,
+                    uint32_t* planes, void* stream);
 
 /* Activations for mpq_conv: x [N][C][H][W] fp32 -> planes[bits][N][H][W][C/32]
  * (channel innermost: bit t of word cw at a pixel is channel 32*cw + t).  One range value.
@@ -109,6 +130,17 @@ int mpq_gemm(const uint32_t* a_planes, int a_bits, const uint32_t* b_planes, int
              int32_t* c_i32, float* c_f32, int64_t ldc,
              const float* a_scale, const float* b_scale, int b_mode, void* stream);
 
+/* mpq_gemm with the glue of a chained layer folded into the store.  f = float(c_i32) * alpha[c]
+ * (Eq. 18); if `bias` (n values, one per output column; the paper's layer has none, Section 3.1)
+ * f = f + bias[c]; if `residual` ([m x n], row stride ldc) f = f + residual[r][c]; if `relu`
+ * f = max(f, 0); c_f32 = f.  One rounded fp32 operation each, in that order.  bias, residual and
+ * relu need c_f32; c_i32, when given, still receives the raw accumulators. */
+int mpq_gemm_fused(const uint32_t* a_planes, int a_bits, const uint32_t* b_planes, int b_bits,
+                   int64_t m, int64_t n, int64_t k,
+                   int32_t* c_i32, float* c_f32, int64_t ldc,
+                   const float* a_scale, const float* b_scale, int b_mode,
+                   const float* bias, const float* residual, int relu, void* stream);
+
 /* ---- Convolution by the same decomposition (Section 3.1 extends it to convolutions),
  * done as an implicit im2col on the packed planes: GEMM row = output pixel (n, oh, ow),
  * GEMM k = (kh, kw, c).  x_planes from mpq_encode_nchw, w_planes and tap_sums from
@@ -134,6 +166,24 @@ int mpq_conv_fused(const uint32_t* x_planes, int a_bits, int N, int C, int H, in
                    int32_t* y_i32, float* y_f32,
                    const float* x_scale, const float* w_scale, int w_mode,
                    const float* residual, int relu, float* out_max, void* stream);
+
+/* mpq_conv_fused that also runs the CONSUMER's Encoder in its store (Fig. 1: the Decoder of one
+ * layer feeding the Encoder of the next), for networks whose ranges are known before the layer
+ * runs: the paper's fixed HReLU range [0,1] (Table 1), or a calibrated constant.  The value f
+ * that mpq_conv_fused would store is quantized exactly as mpq_encode_nchw would quantize it with
+ * range *next_scale, limiter next_act and next_bits bits, and written as
+ * next_planes[next_bits][N][Ho][Wo][O/32] (the layout mpq_encode_nchw gives that tensor), so the
+ * consumer needs neither the fp32 tensor nor an encode pass.  y_f32 may then be NULL (nothing is
+ * stored in fp32); y_i32, residual, relu and out_max keep their meaning.  O must be a multiple of 32.
+ * With next_planes NULL this is mpq_conv_fused. */
+int mpq_conv_encoded(const uint32_t* x_planes, int a_bits, int N, int C, int H, int W,
+                     const uint32_t* w_planes, int w_bits, const int32_t* tap_sums,
+                     int O, int KH, int KW, int stride, int pad,
+                     int32_t* y_i32, float* y_f32,
+                     const float* x_scale, const float* w_scale, int w_mode,
+                     const float* residual, int relu, float* out_max,
+                     const float* next_scale, int next_act, int next_bits, uint32_t* next_planes,
+                     void* stream);
 
 /* Sets `bytes` bytes of device memory to zero on the stream (ranges that kernels raise by atomic maximum). */
 int mpq_zero(void* p, int64_t bytes, void* stream);
@@ -203,6 +253,19 @@ int mpq_linear_host(const float* x_host, const float* w_host, int64_t m, int64_t
                     int a_bits, int w_bits, int a_act, int w_mode,
                     int32_t* out_i32_host, float* out_f32_host,
                     void* workspace, int64_t workspace_bytes, void* stream);
+
+/* The deployed form of mpq_linear_host: the weights were encoded once (mpq_absmax + mpq_encode)
+ * and stay on the device as w_planes [w_bits][n][mpq_row_words(k)] with their range(s) w_scale
+ * (1 or n values); every call moves only the activations up (x_host, [m x k]) and the results
+ * down.  Same pipeline as mpq_linear_host otherwise (row blocks copied back on the helper stream
+ * while the next block is computed; synchronizes `stream`; two calls on one device must not
+ * overlap).  workspace: at least mpq_linear_host_prepared_workspace() bytes, 256-byte aligned. */
+int64_t mpq_linear_host_prepared_workspace(int64_t m, int64_t n, int64_t k, int a_bits);
+int mpq_linear_host_prepared(const float* x_host, const uint32_t* w_planes, const float* w_scale,
+                             int64_t m, int64_t n, int64_t k,
+                             int a_bits, int w_bits, int a_act, int w_mode,
+                             int32_t* out_i32_host, float* out_f32_host,
+                             void* workspace, int64_t workspace_bytes, void* stream);
 
 /* ---- Roofline denominator: measures this GPU's 32-bit population-count issue rate with a
  * register-only loop (no memory traffic) and the SM clock it ran at.  Synchronous.

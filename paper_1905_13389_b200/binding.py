@@ -20,6 +20,7 @@ LIB_PATH = os.path.join(_HERE, "libmpq.so")
 OK = 0
 SCALE_PER_TENSOR, SCALE_PER_ROW = 0, 1
 ACT_HTANH, ACT_HRELU = 0, 1
+ENC_LEVELS, ENC_TRIG = 0, 1
 
 _lib = None
 
@@ -47,10 +48,14 @@ def lib() -> ctypes.CDLL:
         L.mpq_packed_words.restype = i64
         L.mpq_absmax.argtypes = [P, i64, i64, i64, i32, i32, P, P]
         L.mpq_encode.argtypes = [P, i64, i64, i64, P, i32, i32, i32, P, P]
+        L.mpq_encode_with.argtypes = [i32, P, i64, i64, i64, P, i32, i32, i32, P, P]
         L.mpq_encode_nchw.argtypes = [P, i32, i32, i32, i32, P, i32, i32, P, P]
         L.mpq_encode_oihw.argtypes = [P, i32, i32, i32, i32, P, i32, i32, P, P, P]
         L.mpq_gemm.argtypes = [P, i32, P, i32, i64, i64, i64, P, P, i64, P, P, i32, P]
+        L.mpq_gemm_fused.argtypes = [P, i32, P, i32, i64, i64, i64, P, P, i64, P, P, i32, P, P, i32, P]
         L.mpq_conv.argtypes = [P, i32, i32, i32, i32, i32, P, i32, P, i32, i32, i32, i32, i32, P, P, P, P, i32, P]
+        L.mpq_conv_encoded.argtypes = [P, i32, i32, i32, i32, i32, P, i32, P, i32, i32, i32, i32, i32, P, P, P, P, i32,
+                                       P, i32, P, P, i32, i32, P, P]
         L.mpq_add_relu.argtypes = [P, P, P, i64, P]
         L.mpq_stem_conv7x7.argtypes = [P, P, P, i32, i32, i32, i32, P]
         L.mpq_maxpool3x3s2.argtypes = [P, P, i32, i32, i32, i32, P, P]
@@ -64,6 +69,9 @@ def lib() -> ctypes.CDLL:
         L.mpq_linear_host_workspace.argtypes = [i64, i64, i64, i32, i32]
         L.mpq_linear_host_workspace.restype = i64
         L.mpq_linear_host.argtypes = [P, P, i64, i64, i64, i32, i32, i32, i32, P, P, P, i64, P]
+        L.mpq_linear_host_prepared_workspace.argtypes = [i64, i64, i64, i32]
+        L.mpq_linear_host_prepared_workspace.restype = i64
+        L.mpq_linear_host_prepared.argtypes = [P, P, P, i64, i64, i64, i32, i32, i32, i32, P, P, P, i64, P]
         L.mpq_measure_popc_peak.argtypes = [ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double),
                                             ctypes.POINTER(ctypes.c_int), P]
         L.mpq_measure_mix_peak.argtypes = [i32, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double),
@@ -73,7 +81,8 @@ def lib() -> ctypes.CDLL:
                                               ctypes.POINTER(ctypes.c_int), P]
         L.mpq_measure_b1_mma_peak.restype = i32
         for name in ("mpq_absmax", "mpq_encode", "mpq_encode_nchw", "mpq_encode_oihw", "mpq_gemm", "mpq_conv",
-                     "mpq_add_relu", "mpq_stem_conv7x7", "mpq_maxpool3x3s2", "mpq_conv_fused", "mpq_zero", "mpq_linear", "mpq_linear_static", "mpq_linear_host", "mpq_measure_popc_peak"):
+                     "mpq_add_relu", "mpq_stem_conv7x7", "mpq_maxpool3x3s2", "mpq_conv_fused", "mpq_zero", "mpq_linear", "mpq_linear_static", "mpq_linear_host", "mpq_measure_popc_peak",
+                     "mpq_encode_with", "mpq_gemm_fused", "mpq_conv_encoded", "mpq_linear_host_prepared"):
             getattr(L, name).restype = i32
         _lib = L
     return _lib
@@ -135,6 +144,17 @@ def encode(x: torch.Tensor, scale: torch.Tensor, bits: int, mode: int = SCALE_PE
     return out
 
 
+def encode_with(encoder: int, x: torch.Tensor, scale: torch.Tensor, bits: int, mode: int = SCALE_PER_TENSOR,
+                act: int = ACT_HTANH, out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """:func:`encode` with the form of the Encoder selectable: ENC_LEVELS or ENC_TRIG (Eq. 11's sines)."""
+    rows, k = x.shape
+    if out is None:
+        out = torch.empty((bits, rows, row_words(k)), dtype=torch.int32, device=x.device)
+    _check(lib().mpq_encode_with(encoder, _ptr(x, torch.float32), rows, k, k, _ptr(scale, torch.float32), mode, act,
+                                 bits, _ptr(out, torch.int32), _stream()), "mpq_encode_with")
+    return out
+
+
 def encode_nchw(x: torch.Tensor, scale: torch.Tensor, bits: int, act: int = ACT_HTANH,
                 out: Optional[torch.Tensor] = None) -> torch.Tensor:
     """[N][C][H][W] fp32 -> planes [bits][N][H][W][C/32]."""
@@ -170,6 +190,20 @@ def gemm(a_planes: torch.Tensor, a_bits: int, b_planes: torch.Tensor, b_bits: in
     return c_i32, c_f32
 
 
+def gemm_fused(a_planes: torch.Tensor, a_bits: int, b_planes: torch.Tensor, b_bits: int, m: int, n: int, k: int,
+               c_i32: Optional[torch.Tensor] = None, c_f32: Optional[torch.Tensor] = None,
+               a_scale: Optional[torch.Tensor] = None, b_scale: Optional[torch.Tensor] = None,
+               b_mode: int = SCALE_PER_TENSOR, bias: Optional[torch.Tensor] = None,
+               residual: Optional[torch.Tensor] = None, relu: bool = False):
+    """:func:`gemm` with bias, residual and max(., 0) folded into the store."""
+    _check(lib().mpq_gemm_fused(_ptr(a_planes, torch.int32), a_bits, _ptr(b_planes, torch.int32), b_bits, m, n, k,
+                                _ptr(c_i32, torch.int32), _ptr(c_f32, torch.float32), n,
+                                _ptr(a_scale, torch.float32), _ptr(b_scale, torch.float32), b_mode,
+                                _ptr(bias, torch.float32), _ptr(residual, torch.float32), int(relu), _stream()),
+           "mpq_gemm_fused")
+    return c_i32, c_f32
+
+
 def conv(x_planes: torch.Tensor, a_bits: int, N: int, C: int, H: int, W: int,
          w_planes: torch.Tensor, w_bits: int, tap_sums: Optional[torch.Tensor],
          O: int, KH: int, KW: int, stride: int, pad: int,
@@ -200,6 +234,29 @@ def conv_fused(x_planes: torch.Tensor, a_bits: int, N: int, C: int, H: int, W: i
                                 _ptr(residual, torch.float32), int(relu), _ptr(out_max, torch.float32), _stream()),
            "mpq_conv_fused")
     return y_i32, y_f32
+
+
+def conv_encoded(x_planes: torch.Tensor, a_bits: int, N: int, C: int, H: int, W: int,
+                 w_planes: torch.Tensor, w_bits: int, tap_sums: Optional[torch.Tensor],
+                 O: int, KH: int, KW: int, stride: int, pad: int,
+                 y_i32: Optional[torch.Tensor], y_f32: Optional[torch.Tensor],
+                 x_scale: torch.Tensor, w_scale: torch.Tensor, w_mode: int,
+                 residual: Optional[torch.Tensor], relu: bool, out_max: Optional[torch.Tensor],
+                 next_scale: torch.Tensor, next_act: int, next_bits: int,
+                 next_planes: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """:func:`conv_fused` whose store also runs the consumer's Encoder with a range known beforehand:
+    returns next_planes [next_bits][N][Ho][Wo][O/32]; y_f32 may be None."""
+    Ho, Wo = (H + 2 * pad - KH) // stride + 1, (W + 2 * pad - KW) // stride + 1
+    if next_planes is None:
+        next_planes = torch.empty((next_bits, N, Ho, Wo, O // 32), dtype=torch.int32, device=x_planes.device)
+    _check(lib().mpq_conv_encoded(_ptr(x_planes, torch.int32), a_bits, N, C, H, W, _ptr(w_planes, torch.int32), w_bits,
+                                  _ptr(tap_sums, torch.int32), O, KH, KW, stride, pad,
+                                  _ptr(y_i32, torch.int32), _ptr(y_f32, torch.float32),
+                                  _ptr(x_scale, torch.float32), _ptr(w_scale, torch.float32), w_mode,
+                                  _ptr(residual, torch.float32), int(relu), _ptr(out_max, torch.float32),
+                                  _ptr(next_scale, torch.float32), next_act, next_bits,
+                                  _ptr(next_planes, torch.int32), _stream()), "mpq_conv_encoded")
+    return next_planes
 
 
 def zero(t: torch.Tensor) -> torch.Tensor:
@@ -296,6 +353,29 @@ def linear_host(x_host: torch.Tensor, w_host: torch.Tensor, a_bits: int, w_bits:
     _check(lib().mpq_linear_host(hp(x_host), hp(w_host), m, n, k, a_bits, w_bits, a_act, w_mode,
                                  hp(out_i32_host), hp(out_f32_host), workspace.data_ptr(), workspace.numel(),
                                  _stream()), "mpq_linear_host")
+    return out_i32_host, out_f32_host
+
+
+def linear_host_prepared_workspace(m: int, n: int, k: int, a_bits: int) -> int:
+    return int(lib().mpq_linear_host_prepared_workspace(m, n, k, a_bits))
+
+
+def linear_host_prepared(x_host: torch.Tensor, w_planes: torch.Tensor, w_scale: torch.Tensor, n: int,
+                         a_bits: int, w_bits: int, a_act: int = ACT_HTANH, w_mode: int = SCALE_PER_TENSOR,
+                         out_i32_host: Optional[torch.Tensor] = None, out_f32_host: Optional[torch.Tensor] = None,
+                         workspace: Optional[torch.Tensor] = None):
+    """:func:`linear_host` with the weights already packed on the device (encoded once): only the
+    activations go up and the results come down; synchronizes the stream."""
+    m, k = x_host.shape
+    if workspace is None:
+        workspace = torch.empty(linear_host_prepared_workspace(m, n, k, a_bits), dtype=torch.uint8, device=w_planes.device)
+    for t in (x_host, out_i32_host, out_f32_host):
+        if t is not None and (t.is_cuda or not t.is_contiguous()):
+            raise ValueError("host tensors must be contiguous CPU tensors")
+    hp = lambda t: None if t is None else t.data_ptr()
+    _check(lib().mpq_linear_host_prepared(hp(x_host), _ptr(w_planes, torch.int32), _ptr(w_scale, torch.float32),
+                                          m, n, k, a_bits, w_bits, a_act, w_mode, hp(out_i32_host), hp(out_f32_host),
+                                          workspace.data_ptr(), workspace.numel(), _stream()), "mpq_linear_host_prepared")
     return out_i32_host, out_f32_host
 
 

@@ -178,6 +178,49 @@ int host_pipe(HostPipe** out) {
     *out = &hp;
     return MPQ_OK;
 }
+
+// Layout of mpq_linear_host_prepared's workspace: the activations' staging, the results, the
+// activation range and the packed activations (the weights are already resident and packed).
+struct PreparedLayout {
+    int64_t x, out_i32, out_f32, s_a, a_planes, total;
+};
+PreparedLayout prepared_layout(int64_t m, int64_t n, int64_t k, int a_bits) {
+    PreparedLayout L;
+    int64_t off = 0;
+    L.x = off; off += up256(m * k * 4);
+    L.out_i32 = off; off += up256(m * n * 4);
+    L.out_f32 = off; off += up256(m * n * 4);
+    L.s_a = off; off += 256;
+    L.a_planes = off; off += up256(mpq_packed_words(m, k, a_bits) * 4);
+    L.total = off;
+    return L;
+}
+
+// The product in row blocks; each finished block travels to the host on the helper stream while
+// the next one is computed.  Returns after everything has drained.
+int product_to_host(const uint32_t* ap, int a_bits, const uint32_t* wp, int w_bits, int64_t m, int64_t n, int64_t k,
+                    int32_t* oi, float* of, int32_t* out_i32_host, float* out_f32_host,
+                    const float* s_a, const float* s_w, int w_mode, cudaStream_t st) {
+    int rc;
+    HostPipe* hp = nullptr;
+    if ((rc = host_pipe(&hp)) != MPQ_OK) return rc;
+    const int blocks = m >= 1024 ? kHostBlocks : 1;
+    const int64_t per = ((m + blocks - 1) / blocks + 63) / 64 * 64;
+    for (int b = 0; b < blocks; ++b) {
+        const int64_t r0 = (int64_t)b * per;
+        if (r0 >= m) break;
+        const int64_t rows = (r0 + per <= m) ? per : m - r0;
+        if ((rc = gemm_rows(ap, a_bits, wp, w_bits, m, r0, rows, n, k, oi, of, n, s_a, s_w, w_mode, st)) != MPQ_OK) return rc;
+        if (cudaEventRecord(hp->block_done[b], st) != cudaSuccess) return MPQ_ERR_CUDA;
+        if (cudaStreamWaitEvent(hp->copy_stream, hp->block_done[b], 0) != cudaSuccess) return MPQ_ERR_CUDA;
+        const size_t off = (size_t)r0 * n, bytes = (size_t)rows * n * 4;
+        if (oi && cudaMemcpyAsync(out_i32_host + off, oi + off, bytes, cudaMemcpyDeviceToHost, hp->copy_stream) != cudaSuccess) return MPQ_ERR_CUDA;
+        if (of && cudaMemcpyAsync(out_f32_host + off, of + off, bytes, cudaMemcpyDeviceToHost, hp->copy_stream) != cudaSuccess) return MPQ_ERR_CUDA;
+    }
+    if (cudaEventRecord(hp->copies_done, hp->copy_stream) != cudaSuccess) return MPQ_ERR_CUDA;
+    if (cudaStreamWaitEvent(st, hp->copies_done, 0) != cudaSuccess) return MPQ_ERR_CUDA;
+    return cudaStreamSynchronize(st) == cudaSuccess ? MPQ_OK : MPQ_ERR_CUDA;
+}
 }  // namespace
 
 extern "C" int mpq_linear_host(const float* x_host, const float* w_host, int64_t m, int64_t n, int64_t k,
@@ -209,23 +252,35 @@ extern "C" int mpq_linear_host(const float* x_host, const float* w_host, int64_t
     if (cudaMemcpyAsync(x, x_host, (size_t)m * k * 4, cudaMemcpyHostToDevice, st) != cudaSuccess) return MPQ_ERR_CUDA;
     if ((rc = mpq_absmax(x, m, k, k, MPQ_SCALE_PER_TENSOR, a_act, s_a, st)) != MPQ_OK) return rc;
     if ((rc = mpq_encode(x, m, k, k, s_a, MPQ_SCALE_PER_TENSOR, a_act, a_bits, ap, st)) != MPQ_OK) return rc;
-    // the product in row blocks; each finished block is copied out on the helper stream
-    HostPipe* hp = nullptr;
-    if ((rc = host_pipe(&hp)) != MPQ_OK) return rc;
-    const int blocks = m >= 1024 ? kHostBlocks : 1;
-    const int64_t per = ((m + blocks - 1) / blocks + 63) / 64 * 64;
-    for (int b = 0; b < blocks; ++b) {
-        const int64_t r0 = (int64_t)b * per;
-        if (r0 >= m) break;
-        const int64_t rows = (r0 + per <= m) ? per : m - r0;
-        if ((rc = gemm_rows(ap, a_bits, wp, w_bits, m, r0, rows, n, k, oi, of, n, s_a, s_w, w_mode, st)) != MPQ_OK) return rc;
-        if (cudaEventRecord(hp->block_done[b], st) != cudaSuccess) return MPQ_ERR_CUDA;
-        if (cudaStreamWaitEvent(hp->copy_stream, hp->block_done[b], 0) != cudaSuccess) return MPQ_ERR_CUDA;
-        const size_t off = (size_t)r0 * n, bytes = (size_t)rows * n * 4;
-        if (oi && cudaMemcpyAsync(out_i32_host + off, oi + off, bytes, cudaMemcpyDeviceToHost, hp->copy_stream) != cudaSuccess) return MPQ_ERR_CUDA;
-        if (of && cudaMemcpyAsync(out_f32_host + off, of + off, bytes, cudaMemcpyDeviceToHost, hp->copy_stream) != cudaSuccess) return MPQ_ERR_CUDA;
-    }
-    if (cudaEventRecord(hp->copies_done, hp->copy_stream) != cudaSuccess) return MPQ_ERR_CUDA;
-    if (cudaStreamWaitEvent(st, hp->copies_done, 0) != cudaSuccess) return MPQ_ERR_CUDA;
-    return cudaStreamSynchronize(st) == cudaSuccess ? MPQ_OK : MPQ_ERR_CUDA;
+    return product_to_host(ap, a_bits, wp, w_bits, m, n, k, oi, of, out_i32_host, out_f32_host, s_a, s_w, w_mode, st);
+}
+
+extern "C" int64_t mpq_linear_host_prepared_workspace(int64_t m, int64_t n, int64_t k, int a_bits) {
+    if (m <= 0 || n <= 0 || k <= 0 || !bits_ok(a_bits)) return 0;
+    return prepared_layout(m, n, k, a_bits).total;
+}
+
+extern "C" int mpq_linear_host_prepared(const float* x_host, const uint32_t* w_planes, const float* w_scale,
+                                        int64_t m, int64_t n, int64_t k,
+                                        int a_bits, int w_bits, int a_act, int w_mode,
+                                        int32_t* out_i32_host, float* out_f32_host,
+                                        void* workspace, int64_t workspace_bytes, void* stream) {
+    if (!x_host || !w_planes || !workspace || (!out_i32_host && !out_f32_host)) return MPQ_ERR_NULL;
+    if (out_f32_host && !w_scale) return MPQ_ERR_NULL;
+    int rc = linear_args_ok(m, n, k, a_bits, w_bits, a_act, w_mode);
+    if (rc != MPQ_OK) return rc;
+    if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0 || !aligned16(w_planes)) return MPQ_ERR_ALIGN;
+    const PreparedLayout L = prepared_layout(m, n, k, a_bits);
+    if (workspace_bytes < L.total) return MPQ_ERR_WORKSPACE;
+    cudaStream_t st = (cudaStream_t)stream;
+    char* ws = static_cast<char*>(workspace);
+    float* x = reinterpret_cast<float*>(ws + L.x);
+    int32_t* oi = out_i32_host ? reinterpret_cast<int32_t*>(ws + L.out_i32) : nullptr;
+    float* of = out_f32_host ? reinterpret_cast<float*>(ws + L.out_f32) : nullptr;
+    float* s_a = reinterpret_cast<float*>(ws + L.s_a);
+    uint32_t* ap = reinterpret_cast<uint32_t*>(ws + L.a_planes);
+    if (cudaMemcpyAsync(x, x_host, (size_t)m * k * 4, cudaMemcpyHostToDevice, st) != cudaSuccess) return MPQ_ERR_CUDA;
+    if ((rc = mpq_absmax(x, m, k, k, MPQ_SCALE_PER_TENSOR, a_act, s_a, st)) != MPQ_OK) return rc;
+    if ((rc = mpq_encode(x, m, k, k, s_a, MPQ_SCALE_PER_TENSOR, a_act, a_bits, ap, st)) != MPQ_OK) return rc;
+    return product_to_host(ap, a_bits, w_planes, w_bits, m, n, k, oi, of, out_i32_host, out_f32_host, s_a, w_scale, w_mode, st);
 }

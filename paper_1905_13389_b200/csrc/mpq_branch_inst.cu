@@ -1,6 +1,6 @@
 // Instantiates the branch-fused kernels for one held-operand width (compile with -DMPQ_HB=1..8):
 // eight translation units build in parallel and together cover all 64 (a_bits, w_bits) pairs.
-#include "mpq_branch_kernel.cuh"
+#include "mpq_branch_launch.cuh"
 
 #ifndef MPQ_HB
 #error "compile with -DMPQ_HB=<1..8>"

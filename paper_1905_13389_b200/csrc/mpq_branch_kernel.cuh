@@ -47,9 +47,16 @@ struct BranchParams {
     int tap_granules;          // copies per filter tap = Cw / granule
     uint32_t tap_magic;        // ceil(2^32 / tap_granules): copy index / tap_granules by one multiply
     const int32_t* tap_sums;   // [KH*KW][O]
-    const float* residual;     // CONV, optional: added to the scaled output (same layout), one rounded add
-    int relu;                  // CONV: store max(value, 0)
+    const float* bias;         // optional: one value per output channel / column, added first (one rounded add)
+    const float* residual;     // optional: added to the scaled output (same layout as the output), one rounded add
+    int relu;                  // store max(value, 0)
     float* out_max;            // CONV, optional: raised (never lowered) to the largest stored max(value, 0)
+    // CONV, optional: the consumer's Encoder folded into the store.  The value that would be stored
+    // as fp32 is quantized with the consumer's range and written as packed planes
+    // next_planes[next_bits][N][Ho][Wo][O/32] (the layout mpq_encode_nchw produces for that tensor).
+    uint32_t* next_planes;
+    const float* next_scale;   // 1 value: the consumer's range, known before this layer runs
+    int next_bits, next_act;
     int half_tail;             // CONV: the last k-quad of a row holds data in its first two words only
     uint32_t pow2[24];         // pow2[e] = 2^e: branch weights read from the constant bank, so that
                                // "popcount * 2^e + acc" stays one integer multiply-add (FMA pipe)
@@ -69,6 +76,16 @@ __device__ __forceinline__ void cp_async_small(void* smem_dst, const void* gsrc,
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
 template <int N>
 __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory"); }
+
+// fp32 value of one GEMM output: decoder scale (Eq. 18), then the optional glue of a chained layer
+// (bias, residual, max(.,0)), one rounded operation each.
+__device__ __forceinline__ float gemm_store_value(const BranchParams& p, int32_t v, float alpha, int64_t row, int64_t col) {
+    float f = __fmul_rn((float)v, alpha);
+    if (p.bias) f = __fadd_rn(f, __ldg(p.bias + col));
+    if (p.residual) f = __fadd_rn(f, __ldg(p.residual + row * p.ldc + col));
+    if (p.relu) f = fmaxf(f, 0.0f);
+    return f;
+}
 
 // ---- The branch products of one output over one k-quad, with carry-save compression ---------
 // S += sum_{i,j} 2^(i+j) * popcount(h_i xor s_j) over the four words of a k-quad.  The 4*HB*SB
@@ -195,11 +212,23 @@ struct BranchTile {
     // as the product has at most 16 plane pairs; a third resident CTA gives the two integer pipes
     // more warps to interleave (W4A4: 0.92 -> 0.94 of the instruction-mix peak).
     static constexpr int resident(int ts) { return (ts == 4 && HB * SB <= 16) ? 3 : 2; }
+    // 16-byte chunks of one k-group's shared-memory region: its ring, or the 256 x TH x TS partial
+    // sums it parks there at the end, whichever is larger
+    __host__ __device__ static constexpr int group_quads(int ts, int ring_quads) {
+        return ring_quads > TH * ts * 64 ? ring_quads : TH * ts * 64;
+    }
 };
 
-template <int HB, int SB, int TS, int MODE>
-__global__ void __launch_bounds__(256, BranchTile<HB, SB>::resident(TS))
+// KS > 1 (GEMM only): the CTA has KS groups of 256 threads that share the tile and take its k-stages
+// in turn (group g computes stages g, g + KS, ...), each with its own staging ring and its own
+// barrier; at the end the groups' partial sums meet in shared memory and group 0 decodes and
+// stores.  For grids of at most one CTA per multiprocessor (a fully-connected layer at small
+// batch) this doubles the warps that interleave on the two integer pipes without splitting the
+// tile any finer; the sums are integers, so the result is the same bit for bit.
+template <int HB, int SB, int TS, int MODE, int KS = 1>
+__global__ void __launch_bounds__(256 * KS, KS == 1 ? BranchTile<HB, SB>::resident(TS) : 1)
 branch_kernel(const BranchParams p) {
+    static_assert(KS == 1 || MODE == kModeGemm, "k-groups are a GEMM variant");
     using T = BranchTile<HB, SB>;
     constexpr int TH = T::TH, KQ = T::KQ, STAGES = T::STAGES;
     constexpr int BH = 16 * TH, BS = 16 * TS;
@@ -207,7 +236,7 @@ branch_kernel(const BranchParams p) {
     constexpr int S_QUADS = SB * KQ * BS;          // ... streamed operand
     constexpr int STAGE_QUADS = H_QUADS + S_QUADS;
 
-    extern __shared__ uint4 smem[];
+    extern __shared__ uint4 smem_all[];
     __shared__ int row_n[MODE == kModeConv ? BS : 1];      // image index, or -1 for rows past the end
     __shared__ int row_ih0[MODE == kModeConv ? BS : 1];    // top-left input coordinate of the window
     __shared__ int row_iw0[MODE == kModeConv ? BS : 1];
@@ -216,13 +245,22 @@ branch_kernel(const BranchParams p) {
     __shared__ unsigned row_out[MODE == kModeConv ? BS : 1];   // bit t set: filter tap t falls outside the image
 
     chain_entry();
-    const int tid = threadIdx.x;
+    const int grp = KS == 1 ? 0 : (int)threadIdx.x / 256;                 // k-group of this thread
+    const int tid = (int)threadIdx.x - 256 * grp;
+    // the group's own region: its ring, which later parks its partial sums
+    constexpr int GROUP_QUADS = T::group_quads(TS, STAGES * STAGE_QUADS);
+    uint4* smem = smem_all + (size_t)grp * GROUP_QUADS;
+    auto group_sync = [&]() {
+        if (KS == 1) __syncthreads();
+        else asm volatile("bar.sync %0, 256;" ::"r"(1 + grp) : "memory");
+    };
     const int tx = tid & 15, ty = tid >> 4;
     const int64_t s_tiles = ceil_div(p.streamed_rows, BS);
     const int64_t s0 = (int64_t)(blockIdx.x % s_tiles) * BS;
     const int64_t h0 = (int64_t)(blockIdx.x / s_tiles) * BH;
     const int64_t kq_total = p.rw / 4;
-    const int n_iters = (int)ceil_div(kq_total, KQ);
+    const int n_iters_all = (int)ceil_div(kq_total, KQ);
+    const int n_iters = (n_iters_all - grp + KS - 1) / KS;               // k-stages grp, grp + KS, ... are mine
 
     if (MODE == kModeConv) {
         for (int r = tid; r < BS; r += 256) {
@@ -321,16 +359,16 @@ branch_kernel(const BranchParams p) {
 
 #pragma unroll
     for (int s = 0; s < STAGES - 1; ++s) {
-        if (s < n_iters) load_stage(s, (int64_t)s * KQ);
+        if (s < n_iters) load_stage(s, (int64_t)(s * KS + grp) * KQ);
         cp_async_commit();
     }
 
     for (int it = 0; it < n_iters; ++it) {
         cp_async_wait<STAGES - 2>();
-        __syncthreads();
+        group_sync();
         {
             const int nxt = it + STAGES - 1;
-            if (nxt < n_iters) load_stage(nxt % STAGES, (int64_t)nxt * KQ);
+            if (nxt < n_iters) load_stage(nxt % STAGES, (int64_t)(nxt * KS + grp) * KQ);
             cp_async_commit();
         }
         const uint4* hs = smem + (size_t)(it % STAGES) * STAGE_QUADS;
@@ -360,7 +398,7 @@ branch_kernel(const BranchParams p) {
         };
         // the last stage may hold fewer than KQ k-quads of data: skip the rest (they are all zero;
         // a group that is only partly live reads zero-filled quads, which add nothing)
-        const int kq_live = (int)min((int64_t)KQ, kq_total - (int64_t)it * KQ);
+        const int kq_live = (int)min((int64_t)KQ, kq_total - (int64_t)(it * KS + grp) * KQ);
         // (conv only) a short k whose last k-quad is half empty: that quad is computed on two words
         const bool half_tail = MODE == kModeConv && GQ == 1 && p.half_tail && it == n_iters - 1;
         using Full = std::integral_constant<int, 4>;
@@ -382,10 +420,32 @@ branch_kernel(const BranchParams p) {
     }
     cp_async_wait<0>();
 
+    if (KS > 1) {
+        // the groups' partial sums meet in shared memory (each group parks its own in its own ring)
+        group_sync();
+        uint32_t* parked = reinterpret_cast<uint32_t*>(smem);
+        if (grp != 0) {
+#pragma unroll
+            for (int a = 0; a < TH; ++a)
+#pragma unroll
+                for (int b = 0; b < TS; ++b) parked[(a * TS + b) * 256 + tid] = acc[a][b];
+        }
+        __syncthreads();
+        if (grp != 0) return;
+#pragma unroll
+        for (int g = 1; g < KS; ++g) {
+            const uint32_t* theirs = reinterpret_cast<const uint32_t*>(smem_all + (size_t)g * GROUP_QUADS);
+#pragma unroll
+            for (int a = 0; a < TH; ++a)
+#pragma unroll
+                for (int b = 0; b < TS; ++b) acc[a][b] += theirs[(a * TS + b) * 256 + tid];
+        }
+    }
+
     // ---- decoder: acc = L_a L_w k - 2 S, then the fused scale of Eq. 18 -------------------
     constexpr uint32_t LL = (uint32_t)(((1 << HB) - 1) * ((1 << SB) - 1));
     const uint32_t full = LL * (uint32_t)p.k;
-    const bool want_f32 = p.out_f32 != nullptr;
+    const bool want_f32 = p.out_f32 != nullptr || p.next_planes != nullptr;
     // activation bits: GEMM held = A; CONV streamed = x
     constexpr int A_BITS = (MODE == kModeGemm) ? HB : SB;
     constexpr int W_BITS = (MODE == kModeGemm) ? SB : HB;
@@ -406,7 +466,7 @@ branch_kernel(const BranchParams p) {
                 if (row >= p.held_rows) continue;
                 const int32_t v = (int32_t)(full - 2u * acc[a][b]);
                 if (p.out_i32) p.out_i32[row * p.ldc + col] = v;
-                if (want_f32) p.out_f32[row * p.ldc + col] = __fmul_rn((float)v, alpha);
+                if (want_f32) p.out_f32[row * p.ldc + col] = gemm_store_value(p, v, alpha, row, col);
             }
         }
     } else {
@@ -421,11 +481,23 @@ branch_kernel(const BranchParams p) {
                 alpha[a] = __fmul_rn(fa, __fdiv_rn(__ldg(p.w_scale + (p.w_per_row ? o : 0)), Lw));
         }
         float seen_max = 0.0f;
+        // consumer's Encoder in the store: its level indices go through a [pixel][channel] byte tile in the
+        // (drained) staging ring, then one ballot per plane packs 32 channels of a pixel into a word
+        const bool want_planes = p.next_planes != nullptr;
+        unsigned char* code_tile = reinterpret_cast<unsigned char*>(smem);
+        float next_inv = 0.0f, next_half_L = 0.0f, next_lo = 0.0f, next_hi = 0.0f;
+        int next_H = 0;
+        if (want_planes) {
+            next_inv = inverse_scale(__ldg(p.next_scale));
+            next_H = 1 << (p.next_bits - 1);
+            next_half_L = 0.5f * (float)((1 << p.next_bits) - 1);
+            next_lo = (float)(-next_H); next_hi = (float)next_H - 0.5f;
+            __syncthreads();                         // every warp is done reading the last k-stage
+        }
 #pragma unroll
         for (int b = 0; b < TS; ++b) {
             const int r = tx + 16 * b;
             const int n = row_n[r];
-            if (n < 0) continue;
             // taps of this pixel that fall outside the image were staged as all-zero bits, i.e. as the
             // code -L_a; what they added, -L_a * tap_sum[tap][o], is taken out again so they count as 0
             const unsigned outside = row_out[r];
@@ -433,7 +505,7 @@ branch_kernel(const BranchParams p) {
 #pragma unroll
             for (int a = 0; a < TH; ++a) {
                 const int64_t o = h0 + ty + 16 * a;
-                if (o >= p.held_rows) continue;
+                if (n < 0 || o >= p.held_rows) continue;
                 int32_t v = (int32_t)(full - 2u * acc[a][b]);
                 if (outside) {
                     // modular arithmetic: the staged value may leave the int32 range, the corrected one does not
@@ -448,8 +520,38 @@ branch_kernel(const BranchParams p) {
                     float f = __fmul_rn((float)v, alpha[a]);
                     if (p.residual) f = __fadd_rn(f, __ldg(p.residual + idx));
                     if (p.relu) f = fmaxf(f, 0.0f);
-                    p.out_f32[idx] = f;
+                    if (p.out_f32) p.out_f32[idx] = f;
                     seen_max = fmaxf(seen_max, f);
+                    if (want_planes) {
+                        const int u = p.next_act == MPQ_ACT_HRELU
+                                          ? level_index<MPQ_ACT_HRELU>(f, next_inv, next_half_L, next_lo, next_hi, next_H)
+                                          : level_index<MPQ_ACT_HTANH>(f, next_inv, next_half_L, next_lo, next_hi, next_H);
+                        code_tile[r * BH + ty + 16 * a] = (unsigned char)u;
+                    }
+                }
+            }
+        }
+        if (want_planes) {
+            __syncthreads();
+            // (pixel, 32-channel group) pairs of the tile, one per warp and step; lane = channel
+            constexpr int GROUPS = BH >= 32 ? BH / 32 : 1;
+            constexpr int LANES = BH >= 32 ? 32 : BH;          // a 16-channel tile fills half a word
+            const int lane = tid & 31, warp = tid >> 5;
+            const int Ow = p.O / 32;
+            const int64_t plane_words = (int64_t)p.N * hw * Ow;
+            for (int task = warp; task < BS * GROUPS; task += 8) {
+                const int r = task / GROUPS, grp = task % GROUPS;
+                const int n = row_n[r];
+                const int64_t o0 = h0 + 32 * grp;
+                const bool live = n >= 0 && o0 < p.held_rows;      // warp-uniform
+                const unsigned u = (live && lane < LANES) ? code_tile[r * BH + 32 * grp + lane] : 0u;
+                for (int q = 0; q < p.next_bits; ++q) {
+                    const unsigned word = __ballot_sync(0xffffffffu, (u >> q) & 1u);
+                    if (live && lane == q) {
+                        const int64_t at = (int64_t)q * plane_words + ((int64_t)n * hw + row_rem[r]) * Ow + o0 / 32;
+                        if (BH >= 32) p.next_planes[at] = word;
+                        else reinterpret_cast<unsigned short*>(p.next_planes)[2 * at + ((o0 >> 4) & 1)] = (unsigned short)word;
+                    }
                 }
             }
         }
@@ -463,47 +565,19 @@ branch_kernel(const BranchParams p) {
     }
 }
 
-template <int HB, int SB, int TS, int MODE>
+template <int HB, int SB, int TS, int MODE, int KS = 1>
 static int launch_branch(const BranchParams& p, cudaStream_t st) {
     using T = BranchTile<HB, SB>;
     constexpr int BH = 16 * T::TH, BS = 16 * TS;
-    constexpr size_t smem_bytes = (size_t)T::STAGES * (HB * T::KQ * BH + SB * T::KQ * BS) * sizeof(uint4);
-    auto kern = branch_kernel<HB, SB, TS, MODE>;
+    constexpr int ring_quads = T::STAGES * (HB * T::KQ * BH + SB * T::KQ * BS);
+    constexpr size_t smem_bytes = (KS == 1 ? (size_t)ring_quads : (size_t)KS * T::group_quads(TS, ring_quads)) * sizeof(uint4);
+    static_assert(smem_bytes <= 227 * 1024, "shared memory of one CTA");
+    auto kern = branch_kernel<HB, SB, TS, MODE, KS>;
     static PerDeviceOnce configured;   // per instantiation: the attribute belongs to (function, device)
     if (configured.raise_smem_limit(kern, smem_bytes) != MPQ_OK) return MPQ_ERR_CUDA;
     const int64_t blocks = ceil_div(p.streamed_rows, BS) * ceil_div(p.held_rows, BH);
     if (blocks <= 0 || blocks > 0x7fffffffLL) return MPQ_ERR_BAD_SHAPE;
-    return launch_chained(kern, (unsigned)blocks, 256, smem_bytes, st, p);
-}
-
-// Streamed-side tile width (16*TS items): the widest tile has the least shared-memory traffic per
-// population count, but a grid of few large tiles leaves SMs idle in its last wave.  Pick the
-// width with the smallest estimated makespan: waves of (resident CTAs x SM count) tiles, each
-// costing its width times the CTAs that share an SM times a measured per-width inefficiency.
-template <int HB, int SB, int MODE>
-static int launch_auto(const BranchParams& p, cudaStream_t st) {
-    using T = BranchTile<HB, SB>;
-    const int64_t held_tiles = ceil_div(p.held_rows, 16 * T::TH);
-    const int sms = sm_count();
-    if (sms <= 0) return MPQ_ERR_CUDA;
-    // (with 7 or 8 streamed planes the 128-wide tile's loop body outgrows the instruction cache)
-    const double penalty[3] = {SB >= 7 ? 1.10 : 1.00, T::resident(4) == 3 ? 0.98 : 1.05, 1.20};      // TS = 8, 4, 2
-    int best = 0;
-    double best_cost = 0.0;
-    for (int c = 0; c < (MODE == kModeConv ? 2 : 3); ++c) {      // the 32-wide tile never won for a convolution
-        const int ts = 8 >> c;
-        const int per_sm = T::resident(ts);
-        const int64_t slots = (int64_t)per_sm * sms;
-        const int64_t tiles = ceil_div(p.streamed_rows, 16 * ts) * held_tiles;
-        // a grid that fits the resident slots takes one tile time; a longer one its share of waves
-        // plus half a wave of tail; a tile's time grows with its width and with the CTAs sharing the SM
-        const double waves = tiles <= slots ? 1.0 : (double)tiles / (double)slots + 0.5;
-        const double cost = waves * ts * per_sm * penalty[c];
-        if (c == 0 || cost < best_cost) { best = c; best_cost = cost; }
-    }
-    if (best == 0) return launch_branch<HB, SB, 8, MODE>(p, st);
-    if (best == 1) return launch_branch<HB, SB, 4, MODE>(p, st);
-    return launch_branch<HB, SB, 2, kModeGemm>(p, st);
+    return launch_chained(kern, (unsigned)blocks, 256 * KS, smem_bytes, st, p);
 }
 
 // One translation unit per held-operand width instantiates all eight streamed widths.

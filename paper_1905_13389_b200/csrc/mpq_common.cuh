@@ -64,10 +64,17 @@ struct PerDeviceOnce {
 
 // Rows [row0, row0 + rows) of the layer product (mpq_gemm on a row block of A): lets a caller
 // overlap the copy-out of finished rows with the product of the next ones.
+// `glue`: what may ride in the store (bias per column, residual with the output's layout, max(.,0)).
+struct GemmGlue {
+    const float* bias = nullptr;
+    const float* residual = nullptr;
+    bool relu = false;
+};
 int gemm_rows(const uint32_t* a_planes, int a_bits, const uint32_t* b_planes, int b_bits,
               int64_t m_total, int64_t row0, int64_t rows, int64_t n, int64_t k,
               int32_t* c_i32, float* c_f32, int64_t ldc,
-              const float* a_scale, const float* b_scale, int b_mode, cudaStream_t stream);
+              const float* a_scale, const float* b_scale, int b_mode, cudaStream_t stream,
+              const GemmGlue& glue = GemmGlue());
 
 // ---- Chained launches (programmatic dependent launch) --------------------------------------
 // A layer is a chain of short kernels on one stream (range, encode, product, add).  Launched
@@ -82,9 +89,11 @@ int gemm_rows(const uint32_t* a_planes, int a_bits, const uint32_t* b_planes, in
 __device__ __forceinline__ void chain_entry() {
     asm volatile("griddepcontrol.launch_dependents;\n\tgriddepcontrol.wait;\n" ::: "memory");
 }
+// `whole_device`: the grid is exactly one CTA per resident slot of the device (a persistent kernel),
+// so early placement cannot unbalance it and the attribute is set whatever the grid size.
 template <typename... Params, typename... Args>
-inline int launch_chained(void (*kernel)(Params...), unsigned blocks, unsigned threads, size_t smem_bytes,
-                          cudaStream_t st, Args... args) {
+inline int launch_chained_as(bool whole_device, void (*kernel)(Params...), unsigned blocks, unsigned threads,
+                             size_t smem_bytes, cudaStream_t st, Args... args) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(blocks, 1, 1);
     cfg.blockDim = dim3(threads, 1, 1);
@@ -92,7 +101,7 @@ inline int launch_chained(void (*kernel)(Params...), unsigned blocks, unsigned t
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = blocks >= 1024u ? 1 : 0;
+    attr[0].val.programmaticStreamSerializationAllowed = (whole_device || blocks >= 1024u) ? 1 : 0;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     if (cudaLaunchKernelEx(&cfg, kernel, static_cast<Params>(args)...) != cudaSuccess) {
@@ -100,6 +109,11 @@ inline int launch_chained(void (*kernel)(Params...), unsigned blocks, unsigned t
         return MPQ_ERR_CUDA;
     }
     return launch_status();
+}
+template <typename... Params, typename... Args>
+inline int launch_chained(void (*kernel)(Params...), unsigned blocks, unsigned threads, size_t smem_bytes,
+                          cudaStream_t st, Args... args) {
+    return launch_chained_as(false, kernel, blocks, threads, smem_bytes, st, args...);
 }
 
 // 1/s, or 0 when s is not a finite positive number (every code then becomes the level above zero).

@@ -12,51 +12,63 @@ namespace mpq {
 // Non-negative floats order like their bit patterns, so the cross-CTA step is an integer atomicMax.
 // ------------------------------------------------------------------------------------------
 constexpr int kAbsmaxThreads = 256;
-constexpr int kAbsmaxChunk = 8192;  // elements per CTA
+constexpr int kAbsmaxChunk = 8192;  // elements per CTA and step
+constexpr int kAbsmaxPerSm = 4;     // CTAs per multiprocessor: 4 x 32 KiB of loads in flight
 
+// The grid is at most a few CTAs per multiprocessor; every CTA walks the chunks of the tensor in
+// a grid-stride loop, so all multiprocessors finish together whatever the tensor's size.
 template <int ACT, bool VEC4>
-__global__ void __launch_bounds__(kAbsmaxThreads)
+__global__ void __launch_bounds__(kAbsmaxThreads, kAbsmaxPerSm)
 absmax_kernel(const float* __restrict__ x, int64_t k, int64_t ldx, int64_t chunks_per_row,
-              int per_row, float* __restrict__ out) {
+              int64_t total_chunks, int per_row, float* __restrict__ out) {
     chain_entry();
-    const int64_t row = blockIdx.x / chunks_per_row;
-    const int64_t e0 = (blockIdx.x % chunks_per_row) * kAbsmaxChunk;
-    const float* xr = x + row * ldx;
-    const int64_t e1 = min(e0 + (int64_t)kAbsmaxChunk, k);
-    float m = 0.0f;
-    if (VEC4) {
-        // row starts are 16-byte aligned and the chunk start is a multiple of 4 elements
-        const int64_t nvec = (e1 - e0) / 4;
-        const float4* xv = reinterpret_cast<const float4*>(xr + e0);
+    __shared__ float warp_max[kAbsmaxThreads / 32];
+    auto publish = [&](float m, int64_t row) {               // CTA-wide maximum -> one atomic
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+        if ((threadIdx.x & 31) == 0) warp_max[threadIdx.x >> 5] = m;
+        __syncthreads();
+        if (threadIdx.x == 0) {
+#pragma unroll
+            for (int w = 1; w < kAbsmaxThreads / 32; ++w) m = fmaxf(m, warp_max[w]);
+            if (m > 0.0f) atomicMax(reinterpret_cast<int*>(out + row), __float_as_int(m));
+        }
+        __syncthreads();
+    };
+    float running = 0.0f;
+    for (int64_t chunk = blockIdx.x; chunk < total_chunks; chunk += gridDim.x) {
+        const int64_t row = chunk / chunks_per_row;
+        const int64_t e0 = (chunk % chunks_per_row) * kAbsmaxChunk;
+        const float* xr = x + row * ldx;
+        const int64_t e1 = min(e0 + (int64_t)kAbsmaxChunk, k);
+        float m = 0.0f;
+        if (VEC4) {
+            // row starts are 16-byte aligned and the chunk start is a multiple of 4 elements
+            const int64_t nvec = (e1 - e0) / 4;
+            const float4* xv = reinterpret_cast<const float4*>(xr + e0);
 #pragma unroll 8
-        for (int64_t i = threadIdx.x; i < nvec; i += kAbsmaxThreads) {
-            float4 v = __ldg(xv + i);
-            if (ACT == MPQ_ACT_HRELU) {
-                m = fmaxf(m, fmaxf(fmaxf(v.x, v.y), fmaxf(v.z, v.w)));
-            } else {
-                m = fmaxf(m, fmaxf(fmaxf(fabsf(v.x), fabsf(v.y)), fmaxf(fabsf(v.z), fabsf(v.w))));
+            for (int64_t i = threadIdx.x; i < nvec; i += kAbsmaxThreads) {
+                float4 v = __ldg(xv + i);
+                if (ACT == MPQ_ACT_HRELU) {
+                    m = fmaxf(m, fmaxf(fmaxf(v.x, v.y), fmaxf(v.z, v.w)));
+                } else {
+                    m = fmaxf(m, fmaxf(fmaxf(fabsf(v.x), fabsf(v.y)), fmaxf(fabsf(v.z), fabsf(v.w))));
+                }
+            }
+            for (int64_t i = e0 + nvec * 4 + threadIdx.x; i < e1; i += kAbsmaxThreads) {
+                float v = __ldg(xr + i);
+                m = fmaxf(m, ACT == MPQ_ACT_HRELU ? v : fabsf(v));
+            }
+        } else {
+            for (int64_t i = e0 + threadIdx.x; i < e1; i += kAbsmaxThreads) {
+                float v = __ldg(xr + i);
+                m = fmaxf(m, ACT == MPQ_ACT_HRELU ? v : fabsf(v));
             }
         }
-        for (int64_t i = e0 + nvec * 4 + threadIdx.x; i < e1; i += kAbsmaxThreads) {
-            float v = __ldg(xr + i);
-            m = fmaxf(m, ACT == MPQ_ACT_HRELU ? v : fabsf(v));
-        }
-    } else {
-        for (int64_t i = e0 + threadIdx.x; i < e1; i += kAbsmaxThreads) {
-            float v = __ldg(xr + i);
-            m = fmaxf(m, ACT == MPQ_ACT_HRELU ? v : fabsf(v));
-        }
+        if (per_row) publish(m, row);
+        else running = fmaxf(running, m);
     }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
-    __shared__ float warp_max[kAbsmaxThreads / 32];
-    if ((threadIdx.x & 31) == 0) warp_max[threadIdx.x >> 5] = m;
-    __syncthreads();
-    if (threadIdx.x == 0) {
-#pragma unroll
-        for (int w = 1; w < kAbsmaxThreads / 32; ++w) m = fmaxf(m, warp_max[w]);
-        if (m > 0.0f) atomicMax(reinterpret_cast<int*>(out + (per_row ? row : 0)), __float_as_int(m));
-    }
+    if (!per_row) publish(running, 0);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -85,6 +97,45 @@ __device__ __forceinline__ void copy_async_16(void* smem_dst, const void* gsrc) 
 __device__ __forceinline__ void copy_async_wait_all() {
     asm volatile("cp.async.commit_group;\ncp.async.wait_group 0;\n" ::: "memory");
 }
+
+
+// ---- Plane words of 32 elements held by one thread, wide codes (5..8 bits) -------------------
+// LaneWords costs two floating-point-pipe operations per element and PLANE, which makes an 8-bit
+// encoder issue-bound.  For wide codes the level index of every element is taken once (one
+// round-down multiply-add leaves it in the low byte of the result, see LaneWords), the 32 bytes are
+// laid out as eight words W_i = [u_i, u_(8+i), u_(16+i), u_(24+i)] (byte j of word i = element
+// 8 j + i), and the eight 8 x 8 bit blocks that the four byte lanes of W_0..W_7 form are transposed
+// in place by three rounds of masked swaps (distance 1, 2, 4).  Afterwards bit 8 j + i of word b is
+// bit b of element 8 j + i: word b is the plane word.  About five integer operations per element
+// instead of sixteen floating-point ones.
+template <int BITS, int ACT>
+struct LaneBytes {
+    uint32_t t[32];                                // 0x4B000000 + level index, per element
+    __device__ __forceinline__ void set(int e, float z) {
+        const float magic = 8388608.0f + (ACT == MPQ_ACT_HRELU ? (float)(1 << (BITS - 1)) : 0.0f);
+        t[e] = __float_as_uint(__fmaf_rd(z, (float)(1 << BITS), magic));
+    }
+    __device__ __forceinline__ void words(uint32_t (&out)[BITS]) const {
+        uint32_t w[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+            w[i] = __byte_perm(__byte_perm(t[i], t[8 + i], 0x0040), __byte_perm(t[16 + i], t[24 + i], 0x0040), 0x5410);
+#pragma unroll
+        for (int d = 1; d <= 4; d *= 2) {
+            const uint32_t mask = d == 1 ? 0x55555555u : d == 2 ? 0x33333333u : 0x0F0F0F0Fu;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                if ((i & d) == 0) {
+                    const uint32_t x = ((w[i] >> d) ^ w[i + d]) & mask;
+                    w[i + d] ^= x;
+                    w[i] ^= x << d;
+                }
+            }
+        }
+#pragma unroll
+        for (int p = 0; p < BITS; ++p) out[p] = w[p];
+    }
+};
 
 template <int BITS, int ACT>
 __global__ void __launch_bounds__(kEncodeThreads)
@@ -119,21 +170,35 @@ encode_rows_kernel(const float* __restrict__ x, int64_t rows, int64_t k, int64_t
         copy_async_wait_all();
         __syncwarp();
         const float4* own = reinterpret_cast<const float4*>(mine + lane * kStageRow);
-        LaneWords<BITS, ACT> lw;
-        lw.clear();
         float probe = 0.0f;                                 // turns NaN if any element is NaN
-#pragma unroll
-        for (int c = 7; c >= 0; --c) {
-            const float4 v = own[c];
-            if (ACT == MPQ_ACT_HTANH) probe = fmaf(v.x, v.y, fmaf(v.z, v.w, probe));
-            lw.push(level_fraction<BITS, ACT>(v.w, inv, half_L), two);
-            lw.push(level_fraction<BITS, ACT>(v.z, inv, half_L), two);
-            lw.push(level_fraction<BITS, ACT>(v.y, inv, half_L), two);
-            lw.push(level_fraction<BITS, ACT>(v.x, inv, half_L), two);
-        }
         uint32_t word[BITS];
+        if constexpr (BITS >= 5) {
+            LaneBytes<BITS, ACT> lb;
 #pragma unroll
-        for (int p = 0; p < BITS; ++p) word[p] = lw.word(p);
+            for (int c = 0; c < 8; ++c) {
+                const float4 v = own[c];
+                if (ACT == MPQ_ACT_HTANH) probe = fmaf(v.x, v.y, fmaf(v.z, v.w, probe));
+                lb.set(4 * c + 0, level_fraction<BITS, ACT>(v.x, inv, half_L));
+                lb.set(4 * c + 1, level_fraction<BITS, ACT>(v.y, inv, half_L));
+                lb.set(4 * c + 2, level_fraction<BITS, ACT>(v.z, inv, half_L));
+                lb.set(4 * c + 3, level_fraction<BITS, ACT>(v.w, inv, half_L));
+            }
+            lb.words(word);
+        } else {
+            LaneWords<BITS, ACT> lw;
+            lw.clear();
+#pragma unroll
+            for (int c = 7; c >= 0; --c) {
+                const float4 v = own[c];
+                if (ACT == MPQ_ACT_HTANH) probe = fmaf(v.x, v.y, fmaf(v.z, v.w, probe));
+                lw.push(level_fraction<BITS, ACT>(v.w, inv, half_L), two);
+                lw.push(level_fraction<BITS, ACT>(v.z, inv, half_L), two);
+                lw.push(level_fraction<BITS, ACT>(v.y, inv, half_L), two);
+                lw.push(level_fraction<BITS, ACT>(v.x, inv, half_L), two);
+            }
+#pragma unroll
+            for (int p = 0; p < BITS; ++p) word[p] = lw.word(p);
+        }
         if (ACT == MPQ_ACT_HTANH && (probe != probe || inv == 0.0f || inv == __int_as_float(0x7f800000))) {
 #pragma unroll
             for (int p = 0; p < BITS; ++p) word[p] = 0u;
@@ -208,23 +273,39 @@ encode_nchw_kernel(const float* __restrict__ x, int N, int C, int64_t HW,
     const float inv = inverse_scale(__ldg(scale));
 
     const float* base = x + ((n * C + (int64_t)cw * 32) * HW + pixel);
-    LaneWords<BITS, ACT> lw;
-    lw.clear();
     float probe = 0.0f;                                     // turns NaN if any element is NaN
-#pragma unroll
-    for (int c0 = 24; c0 >= 0; c0 -= 8) {
-        float v[8];
-#pragma unroll
-        for (int cc = 0; cc < 8; ++cc) v[cc] = __ldg(base + (int64_t)(c0 + cc) * HW);
-#pragma unroll
-        for (int cc = 7; cc >= 0; --cc) {
-            if (ACT == MPQ_ACT_HTANH && (cc & 1)) probe = fmaf(v[cc], v[cc - 1], probe);
-            lw.push(level_fraction<BITS, ACT>(v[cc], inv, half_L), two);
-        }
-    }
     uint32_t word[BITS];
+    if constexpr (BITS >= 5) {
+        LaneBytes<BITS, ACT> lb;
 #pragma unroll
-    for (int p = 0; p < BITS; ++p) word[p] = lw.word(p);
+        for (int c0 = 0; c0 < 32; c0 += 8) {
+            float v[8];
+#pragma unroll
+            for (int cc = 0; cc < 8; ++cc) v[cc] = __ldg(base + (int64_t)(c0 + cc) * HW);
+#pragma unroll
+            for (int cc = 0; cc < 8; ++cc) {
+                if (ACT == MPQ_ACT_HTANH && (cc & 1)) probe = fmaf(v[cc], v[cc - 1], probe);
+                lb.set(c0 + cc, level_fraction<BITS, ACT>(v[cc], inv, half_L));
+            }
+        }
+        lb.words(word);
+    } else {
+        LaneWords<BITS, ACT> lw;
+        lw.clear();
+#pragma unroll
+        for (int c0 = 24; c0 >= 0; c0 -= 8) {
+            float v[8];
+#pragma unroll
+            for (int cc = 0; cc < 8; ++cc) v[cc] = __ldg(base + (int64_t)(c0 + cc) * HW);
+#pragma unroll
+            for (int cc = 7; cc >= 0; --cc) {
+                if (ACT == MPQ_ACT_HTANH && (cc & 1)) probe = fmaf(v[cc], v[cc - 1], probe);
+                lw.push(level_fraction<BITS, ACT>(v[cc], inv, half_L), two);
+            }
+        }
+#pragma unroll
+        for (int p = 0; p < BITS; ++p) word[p] = lw.word(p);
+    }
     if (ACT == MPQ_ACT_HTANH && (probe != probe || inv == 0.0f || inv == __int_as_float(0x7f800000))) {
 #pragma unroll
         for (int p = 0; p < BITS; ++p) word[p] = 0u;
@@ -350,10 +431,12 @@ extern "C" int mpq_absmax(const float* x, int64_t rows, int64_t k, int64_t ldx, 
     if (cudaMemsetAsync(scale_out, 0, sizeof(float) * (per_row ? rows : 1), st) != cudaSuccess) return MPQ_ERR_CUDA;
     if (!per_row && ldx == k) { k = rows * k; ldx = k; rows = 1; }   // contiguous tensor: one long row
     const int64_t chunks = ceil_div(k, kAbsmaxChunk);
-    const int64_t blocks = rows * chunks;
-    if (blocks > 0x7fffffffLL) return MPQ_ERR_BAD_SHAPE;
+    const int64_t total = rows * chunks;
+    const int sms = sm_count();
+    if (sms <= 0) return MPQ_ERR_CUDA;
+    const int64_t blocks = min(total, (int64_t)sms * kAbsmaxPerSm);
     const bool vec4 = aligned16(x) && (ldx % 4 == 0);
-#define MPQ_LAUNCH(A, V) launch_chained(absmax_kernel<A, V>, (unsigned)blocks, kAbsmaxThreads, 0, st, x, k, ldx, chunks, per_row, scale_out)
+#define MPQ_LAUNCH(A, V) launch_chained_as(blocks == (int64_t)sms * kAbsmaxPerSm, absmax_kernel<A, V>, (unsigned)blocks, kAbsmaxThreads, 0, st, x, k, ldx, chunks, total, per_row, scale_out)
     if (act == MPQ_ACT_HRELU) return vec4 ? MPQ_LAUNCH(MPQ_ACT_HRELU, true) : MPQ_LAUNCH(MPQ_ACT_HRELU, false);
     return vec4 ? MPQ_LAUNCH(MPQ_ACT_HTANH, true) : MPQ_LAUNCH(MPQ_ACT_HTANH, false);
 #undef MPQ_LAUNCH

@@ -1,5 +1,5 @@
 // C-ABI entry points of the layer product: argument checks, then dispatch on the bit-widths.
-#include "mpq_branch_kernel.cuh"
+#include "mpq_branch_launch.cuh"
 
 namespace mpq {
 
@@ -52,9 +52,11 @@ using namespace mpq;
 int mpq::gemm_rows(const uint32_t* a_planes, int a_bits, const uint32_t* b_planes, int b_bits,
                    int64_t m_total, int64_t row0, int64_t rows, int64_t n, int64_t k,
                    int32_t* c_i32, float* c_f32, int64_t ldc,
-                   const float* a_scale, const float* b_scale, int b_mode, cudaStream_t stream) {
+                   const float* a_scale, const float* b_scale, int b_mode, cudaStream_t stream,
+                   const GemmGlue& glue) {
     if (!a_planes || !b_planes || (!c_i32 && !c_f32)) return MPQ_ERR_NULL;
     if (c_f32 && (!a_scale || !b_scale)) return MPQ_ERR_NULL;
+    if ((glue.bias || glue.residual || glue.relu) && !c_f32) return MPQ_ERR_NULL;
     if (m_total <= 0 || n <= 0 || k <= 0 || ldc < n || row0 < 0 || rows <= 0 || row0 + rows > m_total) return MPQ_ERR_BAD_SHAPE;
     if (!bits_ok(a_bits) || !bits_ok(b_bits) ||
         (b_mode != MPQ_SCALE_PER_TENSOR && b_mode != MPQ_SCALE_PER_ROW)) return MPQ_ERR_UNSUPPORTED;
@@ -68,6 +70,9 @@ int mpq::gemm_rows(const uint32_t* a_planes, int a_bits, const uint32_t* b_plane
     p.out_f32 = c_f32 ? c_f32 + row0 * ldc : nullptr;
     p.ldc = ldc;
     p.a_scale = a_scale; p.w_scale = b_scale; p.w_per_row = b_mode == MPQ_SCALE_PER_ROW;
+    p.bias = glue.bias;
+    p.residual = glue.residual ? glue.residual + row0 * ldc : nullptr;
+    p.relu = glue.relu;
     fill_pow2(p);
     return dispatch_gemm(a_bits, b_bits, p, stream);
 }
@@ -78,6 +83,17 @@ extern "C" int mpq_gemm(const uint32_t* a_planes, int a_bits, const uint32_t* b_
                         const float* a_scale, const float* b_scale, int b_mode, void* stream) {
     return mpq::gemm_rows(a_planes, a_bits, b_planes, b_bits, m, 0, m, n, k, c_i32, c_f32, ldc,
                           a_scale, b_scale, b_mode, (cudaStream_t)stream);
+}
+
+extern "C" int mpq_gemm_fused(const uint32_t* a_planes, int a_bits, const uint32_t* b_planes, int b_bits,
+                              int64_t m, int64_t n, int64_t k,
+                              int32_t* c_i32, float* c_f32, int64_t ldc,
+                              const float* a_scale, const float* b_scale, int b_mode,
+                              const float* bias, const float* residual, int relu, void* stream) {
+    GemmGlue glue;
+    glue.bias = bias; glue.residual = residual; glue.relu = relu != 0;
+    return mpq::gemm_rows(a_planes, a_bits, b_planes, b_bits, m, 0, m, n, k, c_i32, c_f32, ldc,
+                          a_scale, b_scale, b_mode, (cudaStream_t)stream, glue);
 }
 
 extern "C" int mpq_conv(const uint32_t* x_planes, int a_bits, int N, int C, int H, int W,
@@ -95,10 +111,29 @@ extern "C" int mpq_conv_fused(const uint32_t* x_planes, int a_bits, int N, int C
                         int32_t* y_i32, float* y_f32,
                         const float* x_scale, const float* w_scale, int w_mode,
                         const float* residual, int relu, float* out_max, void* stream) {
-    if ((residual || relu || out_max) && !y_f32) return MPQ_ERR_NULL;
+    return mpq_conv_encoded(x_planes, a_bits, N, C, H, W, w_planes, w_bits, tap_sums, O, KH, KW, stride, pad,
+                            y_i32, y_f32, x_scale, w_scale, w_mode, residual, relu, out_max,
+                            nullptr, 0, 0, nullptr, stream);
+}
 
-    if (!x_planes || !w_planes || (!y_i32 && !y_f32)) return MPQ_ERR_NULL;
-    if (y_f32 && (!x_scale || !w_scale)) return MPQ_ERR_NULL;
+extern "C" int mpq_conv_encoded(const uint32_t* x_planes, int a_bits, int N, int C, int H, int W,
+                        const uint32_t* w_planes, int w_bits, const int32_t* tap_sums,
+                        int O, int KH, int KW, int stride, int pad,
+                        int32_t* y_i32, float* y_f32,
+                        const float* x_scale, const float* w_scale, int w_mode,
+                        const float* residual, int relu, float* out_max,
+                        const float* next_scale, int next_act, int next_bits, uint32_t* next_planes,
+                        void* stream) {
+    const bool want_f32 = y_f32 || next_planes;
+    if ((residual || relu || out_max) && !want_f32) return MPQ_ERR_NULL;
+    if (!x_planes || !w_planes || (!y_i32 && !want_f32)) return MPQ_ERR_NULL;
+    if (want_f32 && (!x_scale || !w_scale)) return MPQ_ERR_NULL;
+    if (next_planes) {
+        if (!next_scale) return MPQ_ERR_NULL;
+        if (!bits_ok(next_bits) || (next_act != MPQ_ACT_HTANH && next_act != MPQ_ACT_HRELU) || O % 32 != 0)
+            return MPQ_ERR_UNSUPPORTED;
+        if (!aligned16(next_planes)) return MPQ_ERR_ALIGN;
+    }
     if (N <= 0 || C <= 0 || H <= 0 || W <= 0 || O <= 0) return MPQ_ERR_BAD_SHAPE;
     if (!bits_ok(a_bits) || !bits_ok(w_bits) || !((KH == 1 && KW == 1) || (KH == 3 && KW == 3)) ||
         (stride != 1 && stride != 2) || pad < 0 || pad > 1 ||
@@ -126,6 +161,7 @@ extern "C" int mpq_conv_fused(const uint32_t* x_planes, int a_bits, int N, int C
     if ((int64_t)N * H * W >= ((int64_t)1 << 31) || (p.rw << p.granule_shift) >= 65536) return MPQ_ERR_UNSUPPORTED;
     p.tap_sums = tap_sums;
     p.residual = residual; p.relu = relu != 0; p.out_max = out_max;
+    p.next_planes = next_planes; p.next_scale = next_scale; p.next_bits = next_bits; p.next_act = next_act;
     fill_pow2(p);
     p.half_tail = (ceil_div(K, 32) % 4 == 1 || ceil_div(K, 32) % 4 == 2) ? 1 : 0;
     // held = weights (w_bits planes), streamed = activations (a_bits planes)

@@ -14,6 +14,13 @@ one is a single fp32 add + max.  Weights are encoded once, at construction, with
 output channel.  All buffers are allocated at construction; ``forward`` only launches kernels
 on the current stream and never synchronises.
 
+With ``static_ranges`` (a dict: encoded convolution name -> range of its input encoder) the ranges
+are fixed before the network runs -- the paper's own setting, where HReLU limits every activation
+to a known interval (Table 1), or constants calibrated on sample data with ``calibrated_ranges``.
+Then every convolution also runs its consumer's Encoder in its store and writes the packed planes
+directly: a block is  conv, conv (+ shortcut conv)  with no encode pass and no fp32 tensor between
+conv1 and conv2; the block output is still stored in fp32 where the next block adds it as shortcut.
+
 With ``fused=True`` (the default) the glue rides in the convolutions' stores: conv2 adds the
 shortcut and applies max(.,0) itself, and every producer (max-pool, conv1, conv2) raises the
 range of the encoder that consumes it, so a block is  encode, conv, encode, conv (+ shortcut
@@ -56,7 +63,8 @@ class _QConv:
 class QuantResNet18Stack:
     def __init__(self, weights: Dict[str, np.ndarray], batch: int, size: int = 224,
                  a_bits: int = 4, w_bits: int = 4, device: Optional[torch.device] = None,
-                 keep_int32: bool = False, fused: bool = True):
+                 keep_int32: bool = False, fused: bool = True,
+                 static_ranges: Optional[Dict[str, float]] = None):
         dev = device or torch.device("cuda", torch.cuda.current_device())
         self.dev, self.batch, self.size, self.a_bits, self.w_bits = dev, batch, size, a_bits, w_bits
         self.keep_int32 = keep_int32
@@ -103,6 +111,13 @@ class QuantResNet18Stack:
                     self.y_i32[name] = torch.empty((batch, cout, Ho, Ho), dtype=torch.int32, device=dev)
             self.block_out[blk] = f32(batch, cout, Ho, Ho)
             H = Ho
+        self.static = static_ranges is not None
+        if self.static:
+            missing = [n for n in self.x_scale if n not in static_ranges]
+            if missing:
+                raise ValueError("static_ranges lacks %s" % ", ".join(missing))
+            host = torch.tensor([float(static_ranges[n]) for n in self.x_scale], dtype=torch.float32)
+            self.scales.copy_(host.to(dev))                # x_scale[name] are views of this tensor, in this order
         self.layer_names: List[str] = ["stem", "maxpool"]
         for blk, _, _, _, has_ds in BLOCKS:
             self.layer_names += [blk + ".conv1", blk + ".conv2"] + ([blk + ".downsample"] if has_ds else [])
@@ -136,6 +151,8 @@ class QuantResNet18Stack:
             events[name] = (e0, e1)
             return r
 
+        if self.static:
+            return self._forward_static(x, span)
         if self.fused:
             return self._forward_fused(x, span)
         span("stem", lambda: mpq.stem_conv7x7(x, self.stem_w, True, out=self.stem_out))
@@ -186,4 +203,46 @@ class QuantResNet18Stack:
                 p = mpq.encode_nchw(t, s2, self.a_bits, mpq.ACT_HRELU, out=self.x_planes[n2])
                 return self._conv_fused(n2, p, s2, self.block_out[blk], shortcut, True, next_scale)
             cur = span(n2, second)
+        return cur
+
+    def calibrated_ranges(self) -> Dict[str, float]:
+        """The ranges the encoders saw in the last (non-static) forward, as ``static_ranges`` input."""
+        vals = self.scales.cpu().tolist()
+        return {name: vals[i] for i, name in enumerate(self.x_scale)}
+
+    def _conv_encoded(self, name, planes, scale, out, residual, relu, next_name):
+        """Convolution `name`; with `next_name` its store also writes that consumer's packed planes."""
+        c = self.convs[name]
+        C, H, W = self.in_shape[name]
+        if next_name is None:
+            mpq.conv_fused(planes, self.a_bits, self.batch, C, H, W, c.w_planes, self.w_bits, c.tap_sums,
+                           c.O, c.KH, c.KW, c.stride, c.pad, self.y_i32.get(name), out,
+                           scale, c.w_scale, mpq.SCALE_PER_ROW, residual, relu, None)
+        else:
+            mpq.conv_encoded(planes, self.a_bits, self.batch, C, H, W, c.w_planes, self.w_bits, c.tap_sums,
+                             c.O, c.KH, c.KW, c.stride, c.pad, self.y_i32.get(name), out,
+                             scale, c.w_scale, mpq.SCALE_PER_ROW, residual, relu, None,
+                             self.x_scale[next_name], mpq.ACT_HRELU, self.a_bits, self.x_planes[next_name])
+        return out
+
+    def _forward_static(self, x, span):
+        span("stem", lambda: mpq.stem_conv7x7(x, self.stem_w, True, out=self.stem_out))
+        cur = span("maxpool", lambda: mpq.maxpool3x3s2(self.stem_out, out=self.pooled))
+        first = BLOCKS[0][0] + ".conv1"
+        span("encode", lambda: mpq.encode_nchw(cur, self.x_scale[first], self.a_bits, mpq.ACT_HRELU, out=self.x_planes[first]))
+        for bi, (blk, cin, cout, stride, has_ds) in enumerate(BLOCKS):
+            n1, n2, nd = blk + ".conv1", blk + ".conv2", blk + ".downsample"
+            last = bi + 1 == len(BLOCKS)
+            next_n1 = None if last else BLOCKS[bi + 1][0] + ".conv1"
+            next_has_ds = (not last) and BLOCKS[bi + 1][4]
+            # conv1 feeds conv2 only: no fp32 tensor, just conv2's planes
+            span(n1, lambda: self._conv_encoded(n1, self.x_planes[n1], self.x_scale[n1], None, None, False, n2))
+            shortcut = span(nd, lambda: self._conv_encoded(nd, self.x_planes[n1], self.x_scale[n1], self.y[nd], None, False, None)) \
+                if has_ds else cur
+            # conv2 adds the shortcut, applies max(.,0) and writes the next block's planes; its fp32 output is
+            # kept only where somebody adds it later (the next block's shortcut) or reads it (the last block)
+            keep = last or not next_has_ds
+            out = self.block_out[blk] if keep else None
+            span(n2, lambda: self._conv_encoded(n2, self.x_planes[n2], self.x_scale[n2], out, shortcut, True, next_n1))
+            cur = self.block_out[blk]
         return cur

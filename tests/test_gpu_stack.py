@@ -130,3 +130,50 @@ def test_stack_repeated_forwards_are_identical(mpq, cuda):
     torch.cuda.synchronize()
     assert torch.equal(out, first) and torch.equal(net.scales, scales)
     assert float(scales.min()) > 0
+
+
+@pytest.mark.parametrize("a_bits,w_bits", [(4, 4), (3, 5)])
+def test_stack_static_ranges_write_planes_from_the_store(mpq, cuda, a_bits, w_bits):
+    """Ranges fixed before the network runs (here: calibrated on the same batch, so the codes must be
+    the dynamic run's): every convolution writes its consumer's packed planes from its store, there is
+    no encode pass after the first one and no fp32 tensor between conv1 and conv2 -- and the output,
+    every accumulator and every plane word equal the dynamic run's, which the oracle pins."""
+    batch, size = 2, 64
+    ws = inputs.config5_weights()
+    x = torch.from_numpy(inputs.config5_input(batch, size)).to(cuda)
+    dyn = QuantResNet18Stack(ws, batch, size, a_bits, w_bits, cuda, keep_int32=True, fused=True)
+    ref = dyn.forward(x).clone()
+    torch.cuda.synchronize()
+    ranges = dyn.calibrated_ranges()
+    assert len(ranges) == 16 and min(ranges.values()) > 0
+    net = QuantResNet18Stack(ws, batch, size, a_bits, w_bits, cuda, keep_int32=True, static_ranges=ranges)
+    for t in net.y.values():
+        t.fill_(float("nan"))                                 # nothing may depend on the fp32 intermediates
+    out = net.forward(x)
+    torch.cuda.synchronize()
+    assert torch.equal(out, ref)
+    for name in dyn.y_i32:
+        assert torch.equal(net.y_i32[name], dyn.y_i32[name]), name
+    for name in dyn.x_planes:
+        assert torch.equal(net.x_planes[name], dyn.x_planes[name]), name
+    for blk, _, _, _, _ in BLOCKS:
+        assert bool(torch.isnan(net.y[blk + ".conv1"]).all())  # conv1 -> conv2 went through planes only
+    # the paper's own setting: one fixed range for every encoder (HReLU to [0, s]); the chain still
+    # equals the oracle's chain with that range, block by block
+    fixed = {n: 2.0 for n in ranges}
+    net2 = QuantResNet18Stack(ws, batch, size, a_bits, w_bits, cuda, keep_int32=True, static_ranges=fixed)
+    out2 = net2.forward(x).cpu().numpy()
+    cur = net2.pooled.cpu().numpy()
+    s = np.array([2.0], np.float32)
+    for blk, _, _, stride, has_ds in BLOCKS:
+        qx = oracle.quantize(cur, s, a_bits, act=oracle.HRELU)
+        def conv(name, q, st, pad):
+            s_w = oracle.absmax(ws[name], True)
+            acc = oracle.conv(q, oracle.quantize(ws[name], s_w, w_bits, per_row=True), st, pad)
+            assert np.array_equal(net2.y_i32[name].cpu().numpy(), acc), name
+            return oracle.scale(acc, s[0], s_w, a_bits, w_bits)
+        t = conv(blk + ".conv1", qx, stride, 1)
+        u = conv(blk + ".conv2", oracle.quantize(t, s, a_bits, act=oracle.HRELU), 1, 1)
+        sc = conv(blk + ".downsample", qx, stride, 0) if has_ds else cur
+        cur = oracle.epilogue(u, None, sc, True)
+    assert np.array_equal(out2, cur)
