@@ -13,7 +13,7 @@ namespace mpq {
 // ------------------------------------------------------------------------------------------
 constexpr int kAbsmaxThreads = 256;
 constexpr int kAbsmaxChunk = 8192;  // elements per CTA and step
-constexpr int kAbsmaxPerSm = 4;     // CTAs per multiprocessor: 4 x 32 KiB of loads in flight
+constexpr int kAbsmaxPerSm = 6;     // CTAs per multiprocessor: 6 x 32 KiB of loads in flight
 
 // The grid is at most a few CTAs per multiprocessor; every CTA walks the chunks of the tensor in
 // a grid-stride loop, so all multiprocessors finish together whatever the tensor's size.
@@ -46,13 +46,21 @@ absmax_kernel(const float* __restrict__ x, int64_t k, int64_t ldx, int64_t chunk
             // row starts are 16-byte aligned and the chunk start is a multiple of 4 elements
             const int64_t nvec = (e1 - e0) / 4;
             const float4* xv = reinterpret_cast<const float4*>(xr + e0);
-#pragma unroll 8
-            for (int64_t i = threadIdx.x; i < nvec; i += kAbsmaxThreads) {
-                float4 v = __ldg(xv + i);
-                if (ACT == MPQ_ACT_HRELU) {
-                    m = fmaxf(m, fmaxf(fmaxf(v.x, v.y), fmaxf(v.z, v.w)));
-                } else {
-                    m = fmaxf(m, fmaxf(fmaxf(fabsf(v.x), fabsf(v.y)), fmaxf(fabsf(v.z), fabsf(v.w))));
+            // eight 16-byte loads of every thread are issued before the first one is used
+            for (int64_t i0 = threadIdx.x; i0 < nvec; i0 += 8 * kAbsmaxThreads) {
+                float4 v[8];
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const int64_t i = i0 + j * kAbsmaxThreads;
+                    v[j] = i < nvec ? __ldcs(xv + i) : make_float4(0.0f, 0.0f, 0.0f, 0.0f);   // read once: streaming load
+                }
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    if (ACT == MPQ_ACT_HRELU) {
+                        m = fmaxf(m, fmaxf(fmaxf(v[j].x, v[j].y), fmaxf(v[j].z, v[j].w)));
+                    } else {
+                        m = fmaxf(m, fmaxf(fmaxf(fabsf(v[j].x), fabsf(v[j].y)), fmaxf(fabsf(v[j].z), fabsf(v[j].w))));
+                    }
                 }
             }
             for (int64_t i = e0 + nvec * 4 + threadIdx.x; i < e1; i += kAbsmaxThreads) {
@@ -108,6 +116,7 @@ __device__ __forceinline__ void copy_async_wait_all() {
 // in place by three rounds of masked swaps (distance 1, 2, 4).  Afterwards bit 8 j + i of word b is
 // bit b of element 8 j + i: word b is the plane word.  About five integer operations per element
 // instead of sixteen floating-point ones.
+constexpr int kByteBuilderFromBits = 3;       // narrower codes keep LaneWords (measured)
 template <int BITS, int ACT>
 struct LaneBytes {
     uint32_t t[32];                                // 0x4B000000 + level index, per element
@@ -172,7 +181,7 @@ encode_rows_kernel(const float* __restrict__ x, int64_t rows, int64_t k, int64_t
         const float4* own = reinterpret_cast<const float4*>(mine + lane * kStageRow);
         float probe = 0.0f;                                 // turns NaN if any element is NaN
         uint32_t word[BITS];
-        if constexpr (BITS >= 5) {
+        if constexpr (BITS >= kByteBuilderFromBits) {
             LaneBytes<BITS, ACT> lb;
 #pragma unroll
             for (int c = 0; c < 8; ++c) {
@@ -246,12 +255,16 @@ encode_rows_kernel(const float* __restrict__ x, int64_t rows, int64_t k, int64_t
 }
 
 // ------------------------------------------------------------------------------------------
-// NCHW activations -> planes[bits][N][H][W][C/32].  A warp takes 32 pixels x 32 channels:
-// lane = pixel, so each of the 32 channel reads is a coalesced 128-byte row of one channel,
-// and every lane builds the word of its own pixel (channel c -> bit c) with LaneWords.
+// NCHW activations -> planes[bits][N][H][W][C/32].  A warp takes 32 pixels x G adjacent channel
+// words (G = 1, 2 or 4: all of them for C = 32 and 64): lane = pixel, so each channel read is a
+// coalesced 128-byte row of one channel -- the 32 reads of a word are all in flight together --
+// and every lane builds the G words of its own pixel (channel c -> bit c) and stores them as one
+// 4-, 8- or 16-byte vector, so that the warp's stores cover whole 32-byte sectors.
 // ------------------------------------------------------------------------------------------
-template <int BITS, int ACT>
-__global__ void __launch_bounds__(kEncodeThreads)
+constexpr int kNchwPerSm = 3;          // 80 registers per thread: 32 loads in flight and the words built so far
+
+template <int BITS, int ACT, int G>
+__global__ void __launch_bounds__(kEncodeThreads, kNchwPerSm)
 encode_nchw_kernel(const float* __restrict__ x, int N, int C, int64_t HW,
                    const float* __restrict__ scale, uint32_t* __restrict__ planes,
                    int64_t pix_blocks, int64_t total_warps, uint32_t two) {
@@ -260,10 +273,11 @@ encode_nchw_kernel(const float* __restrict__ x, int N, int C, int64_t HW,
     if (warp >= total_warps) return;
     const int lane = threadIdx.x & 31;
     const int Cw = C / 32;
+    const int groups = Cw / G;
     const int64_t pb = warp % pix_blocks;
     const int64_t rest = warp / pix_blocks;
-    const int cw = (int)(rest % Cw);
-    const int64_t n = rest / Cw;
+    const int cw0 = (int)(rest % groups) * G;
+    const int64_t n = rest / groups;
     const int64_t pixel = pb * 32 + lane;
     if (pixel >= HW) return;
 
@@ -272,52 +286,48 @@ encode_nchw_kernel(const float* __restrict__ x, int N, int C, int64_t HW,
     const float lo = (float)(-H), hi = (float)H - 0.5f;
     const float inv = inverse_scale(__ldg(scale));
 
-    const float* base = x + ((n * C + (int64_t)cw * 32) * HW + pixel);
-    float probe = 0.0f;                                     // turns NaN if any element is NaN
-    uint32_t word[BITS];
-    if constexpr (BITS >= 5) {
-        LaneBytes<BITS, ACT> lb;
+    uint32_t word[G][BITS];
 #pragma unroll
-        for (int c0 = 0; c0 < 32; c0 += 8) {
-            float v[8];
+    for (int g = 0; g < G; ++g) {
+        const float* base = x + ((n * C + (int64_t)(cw0 + g) * 32) * HW + pixel);
+        float v[32];
 #pragma unroll
-            for (int cc = 0; cc < 8; ++cc) v[cc] = __ldg(base + (int64_t)(c0 + cc) * HW);
+        for (int c = 0; c < 32; ++c) v[c] = __ldg(base + (int64_t)c * HW);
+        float probe = 0.0f;                                 // turns NaN if any element is NaN
+        if (ACT == MPQ_ACT_HTANH) {
 #pragma unroll
-            for (int cc = 0; cc < 8; ++cc) {
-                if (ACT == MPQ_ACT_HTANH && (cc & 1)) probe = fmaf(v[cc], v[cc - 1], probe);
-                lb.set(c0 + cc, level_fraction<BITS, ACT>(v[cc], inv, half_L));
-            }
+            for (int c = 0; c < 32; c += 2) probe = fmaf(v[c], v[c + 1], probe);
         }
-        lb.words(word);
-    } else {
-        LaneWords<BITS, ACT> lw;
-        lw.clear();
+        if constexpr (BITS >= kByteBuilderFromBits) {
+            LaneBytes<BITS, ACT> lb;
 #pragma unroll
-        for (int c0 = 24; c0 >= 0; c0 -= 8) {
-            float v[8];
+            for (int c = 0; c < 32; ++c) lb.set(c, level_fraction<BITS, ACT>(v[c], inv, half_L));
+            lb.words(word[g]);
+        } else {
+            LaneWords<BITS, ACT> lw;
+            lw.clear();
 #pragma unroll
-            for (int cc = 0; cc < 8; ++cc) v[cc] = __ldg(base + (int64_t)(c0 + cc) * HW);
+            for (int c = 31; c >= 0; --c) lw.push(level_fraction<BITS, ACT>(v[c], inv, half_L), two);
 #pragma unroll
-            for (int cc = 7; cc >= 0; --cc) {
-                if (ACT == MPQ_ACT_HTANH && (cc & 1)) probe = fmaf(v[cc], v[cc - 1], probe);
-                lw.push(level_fraction<BITS, ACT>(v[cc], inv, half_L), two);
-            }
+            for (int p = 0; p < BITS; ++p) word[g][p] = lw.word(p);
         }
+        if (ACT == MPQ_ACT_HTANH && (probe != probe || inv == 0.0f || inv == __int_as_float(0x7f800000))) {
 #pragma unroll
-        for (int p = 0; p < BITS; ++p) word[p] = lw.word(p);
-    }
-    if (ACT == MPQ_ACT_HTANH && (probe != probe || inv == 0.0f || inv == __int_as_float(0x7f800000))) {
+            for (int p = 0; p < BITS; ++p) word[g][p] = 0u;
+            for (int c = 0; c < 32; ++c) {
+                const uint32_t u = (uint32_t)level_index<ACT>(__ldg(base + (int64_t)c * HW), inv, half_L, lo, hi, H);
 #pragma unroll
-        for (int p = 0; p < BITS; ++p) word[p] = 0u;
-        for (int c = 0; c < 32; ++c) {
-            const uint32_t u = (uint32_t)level_index<ACT>(__ldg(base + (int64_t)c * HW), inv, half_L, lo, hi, H);
-#pragma unroll
-            for (int p = 0; p < BITS; ++p) word[p] |= ((u >> p) & 1u) << c;
+                for (int p = 0; p < BITS; ++p) word[g][p] |= ((u >> p) & 1u) << c;
+            }
         }
     }
 #pragma unroll
-    for (int p = 0; p < BITS; ++p)
-        planes[(((int64_t)p * N + n) * HW + pixel) * Cw + cw] = word[p];
+    for (int p = 0; p < BITS; ++p) {
+        uint32_t* dst = planes + (((int64_t)p * N + n) * HW + pixel) * Cw + cw0;     // G words: G * 4-byte aligned
+        if constexpr (G == 4) *reinterpret_cast<uint4*>(dst) = make_uint4(word[0][p], word[1][p], word[2][p], word[3][p]);
+        else if constexpr (G == 2) *reinterpret_cast<uint2*>(dst) = make_uint2(word[0][p], word[1][p]);
+        else dst[0] = word[0][p];
+    }
 }
 
 // ------------------------------------------------------------------------------------------
@@ -406,13 +416,19 @@ struct EncodeRowsLauncher {
 
 template <int BITS, int ACT>
 struct EncodeNchwLauncher {
-    static int run(const float* x, int N, int C, int64_t HW, const float* scale, uint32_t* planes, cudaStream_t st) {
+    template <int G>
+    static int go(const float* x, int N, int C, int64_t HW, const float* scale, uint32_t* planes, cudaStream_t st) {
         const int64_t pix_blocks = ceil_div(HW, 32);
-        const int64_t warps = pix_blocks * (C / 32) * N;
+        const int64_t warps = pix_blocks * (C / 32 / G) * N;
         const int64_t blocks = ceil_div(warps, kEncodeThreads / 32);
         if (blocks > 0x7fffffffLL) return MPQ_ERR_BAD_SHAPE;
-        return launch_chained(encode_nchw_kernel<BITS, ACT>, (unsigned)blocks, kEncodeThreads, 0, st,
+        return launch_chained(encode_nchw_kernel<BITS, ACT, G>, (unsigned)blocks, kEncodeThreads, 0, st,
                               x, N, C, HW, scale, planes, pix_blocks, warps, 2u);
+    }
+    static int run(const float* x, int N, int C, int64_t HW, const float* scale, uint32_t* planes, cudaStream_t st) {
+        // C is 32, 64 or a multiple of 128 (checked by the caller): 1, 2 or 4 words per lane
+        return C == 32 ? go<1>(x, N, C, HW, scale, planes, st)
+             : C == 64 ? go<2>(x, N, C, HW, scale, planes, st) : go<4>(x, N, C, HW, scale, planes, st);
     }
 };
 
