@@ -11,7 +11,7 @@ import numpy as np
 import torch
 
 from paper_1905_13389_b200 import binding as mpq
-from paper_1905_13389_b200 import inputs
+from paper_1905_13389_b200 import context, inputs
 from paper_1905_13389_b200.resnet18 import QuantResNet18Stack
 
 
@@ -100,6 +100,24 @@ def run_suite(dev: torch.device, hbm_gbs: float, path=None):
         del qa, qb
     except Exception as exc:                                    # library kernel unavailable: the context line is dropped
         out["context_library_int8_gemm_4096"] = {"unavailable": str(exc)[:200]}
+    # context only: this repository's own decoded-integer tensor-core kernel (tcgen05 kind::i8, TMA, TMEM) on the
+    # same shape -- signed form (codes up to 7 bits) and unsigned form with Eq. 17's correction (8-bit codes)
+    qa = torch.randint(-3, 4, (size, size), dtype=torch.int8, device=dev)
+    qb = torch.randint(-3, 4, (size, size), dtype=torch.int8, device=dev)
+    co = torch.empty((size, size), dtype=torch.int32, device=dev)
+    err = torch.zeros(1, dtype=torch.int32, device=dev)
+    ms = _events_ms(lambda: context.i8_gemm(qa, qb, co, err), 10, 3)
+    ua = torch.randint(0, 256, (size, size), dtype=torch.uint8, device=dev)
+    ub = torch.randint(0, 256, (size, size), dtype=torch.uint8, device=dev)
+    sa8, sb8 = context.row_sums_u8(ua), context.row_sums_u8(ub)
+    ms_u = _events_ms(lambda: context.i8_gemm(ua, ub, co, err, unsigned_levels=(255, 255), sums=(sa8, sb8)), 10, 3)
+    out["context_own_tcgen05_i8_gemm_4096"] = {
+        "signed_ms": ms, "signed_tops": 2.0 * size ** 3 / (ms * 1e-3) / 1e12,
+        "unsigned_eq17_ms": ms_u, "unsigned_eq17_tops": 2.0 * size ** 3 / (ms_u * 1e-3) / 1e12,
+        "bounded_wait_ran_out": int(err.cpu()[0]),
+        "note": "decoded-integer product on the 5th-generation tensor cores, own kernel (128 x 128 tile, one CTA per SM, "
+                "no multicast); context for the bit-plane numbers, not part of the library"}
+    del qa, qb, ua, ub, co
 
     # ---- encoders on the sweep's operands (64 MiB fp32 each; four buffers in rotation) ----------
     xs = [x, w, torch.randn_like(x), torch.randn_like(x)]
@@ -248,6 +266,11 @@ def compact(d: dict) -> dict:
         "layers": {n: ([r3(r["ms"]), r3(r["frac_of_branch_peak"])] if "frac_of_branch_peak" in r else [r3(r["ms"])])
                    for n, r in s["layers"].items()},
         "layers_key": "[ms] or [ms, frac of mix peak]"}
+    own = d.get("context_own_tcgen05_i8_gemm_4096", {})
+    if "signed_ms" in own:
+        c["context_int8_tensor_core_gemm_4096"] = {"own_tcgen05_ms": r3(own["signed_ms"]), "own_tcgen05_tops": round(own["signed_tops"], 1),
+                                                   "own_tcgen05_unsigned_eq17_ms": r3(own["unsigned_eq17_ms"]),
+                                                   "library_ms": r3(d.get("context_library_int8_gemm_4096", {}).get("ms", float("nan")))}
     c["encoders"] = {n: {"us": r3(r["us"]), "gb_s": round(r["gb_s"], 1), "frac_of_hbm": r3(r["frac_of_hbm"])}
                      for n, r in d["encoders"].items()}
     return c
@@ -270,6 +293,11 @@ def summary_markdown(d: dict) -> str:
     if "ms" in ctx:
         L.append("\nContext only (not this path): a library int8 tensor-core GEMM of the decoded integers, same shape: "
                  "%.3f ms = %.0f TOPS." % (ctx["ms"], ctx["tops"]))
+    own = d.get("context_own_tcgen05_i8_gemm_4096", {})
+    if "signed_ms" in own:
+        L.append("Own tcgen05 kind::i8 kernel (context, not the library's path): signed codes %.3f ms = %.0f TOPS; 8-bit level "
+                 "indices with the Eq. 17 correction %.3f ms = %.0f TOPS."
+                 % (own["signed_ms"], own["signed_tops"], own["unsigned_eq17_ms"], own["unsigned_eq17_tops"]))
     L += ["\n## Other products\n", "| workload | time | equivalent TOPS | frac of mix peak | frac of plain POPC pipe |",
           "|---|---|---|---|---|",
           "| GEMM W2A2 64x64x512 (int32 + fp32 out) | %.1f us | launch-latency bound | – | – |" % d["gemm_w2a2_64x64x512"]["us"]]

@@ -11,6 +11,9 @@ CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(os.path.dirname(HERE), "include")
 OBJ_DIR = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libmpq.so")
+# context only, never linked into libmpq.so: the decoded-integer tensor-core comparison kernel
+CONTEXT_SRC = os.path.join(CSRC, "context_i8_gemm.cu")
+CONTEXT_LIB = os.path.join(HERE, "libmpq_context.so")
 
 NVCC = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
 ARCH = ["-gencode", "arch=compute_100a,code=sm_100a"]
@@ -62,6 +65,11 @@ def build(force: bool = False, verbose: bool = False) -> str:
         r = subprocess.run(cmd, capture_output=True, text=True)
         if r.returncode != 0:
             raise RuntimeError("link failed:\n%s\n%s" % (r.stdout, r.stderr))
+    if force or not os.path.exists(CONTEXT_LIB) or os.path.getmtime(CONTEXT_LIB) < os.path.getmtime(CONTEXT_SRC):
+        cmd = [NVCC] + ARCH + ["-O3", "-std=c++17", "-lineinfo", "-Xcompiler", "-fPIC", "-shared", "-o", CONTEXT_LIB, CONTEXT_SRC]
+        r = subprocess.run(cmd, capture_output=True, text=True)
+        if r.returncode != 0:
+            raise RuntimeError("nvcc failed for %s:\n%s\n%s" % (CONTEXT_SRC, r.stdout, r.stderr))
     return LIB
 
 

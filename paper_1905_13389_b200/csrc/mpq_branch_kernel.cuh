@@ -274,10 +274,15 @@ branch_kernel(const BranchParams p) {
                 row_iw0[r] = (rem % p.Wo) * p.stride - p.pad;
                 row_pix[r] = (n * p.H + row_ih0[r]) * p.W + row_iw0[r];
                 row_rem[r] = rem;
-                unsigned outside = 0;
-                for (int t = 0; t < p.KH * p.KW; ++t) {
-                    const int ih = row_ih0[r] + t / p.KW, iw = row_iw0[r] + t % p.KW;
-                    if (ih < 0 || ih >= p.H || iw < 0 || iw >= p.W) outside |= 1u << t;
+                // taps outside the image, bit t = tap (t / KW, t % KW).  With padding of at most one pixel only
+                // the first / last row and column of a 3 x 3 window can stick out: whole rows or columns of taps
+                const int ih0 = row_ih0[r], iw0 = row_iw0[r];
+                unsigned outside;
+                if (p.KH == 3) {
+                    outside = (ih0 < 0 ? 0x007u : 0u) | (ih0 + 2 >= p.H ? 0x1C0u : 0u) |
+                              (iw0 < 0 ? 0x049u : 0u) | (iw0 + 2 >= p.W ? 0x124u : 0u);
+                } else {
+                    outside = (ih0 < 0 || ih0 >= p.H || iw0 < 0 || iw0 >= p.W) ? 1u : 0u;
                 }
                 row_out[r] = outside;
             } else {
