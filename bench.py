@@ -35,9 +35,9 @@ SIZE = 4096
 A_BITS = W_BITS = 2
 HBM_FALLBACK_GBS = 6650.0      # used only when MEASURED_PEAKS.json is absent
 # DRAM bytes per launch of the GEMM kernel (dram__bytes_read.sum + dram__bytes_write.sum) from the
-# kept ncu capture of this command: 8.46 MB + 80.40 MB.
+# kept ncu capture of this command: 8.48 MB + 79.9 MB.
 # Set back to None whenever branch_kernel changes after that capture.
-GEMM_DRAM_TRAFFIC_BYTES = 88.9e6
+GEMM_DRAM_TRAFFIC_BYTES = 88.4e6
 ORACLE_SAMPLE_ROWS = 1024      # activation rows of the bounded sample the CPU oracle is timed on
 
 

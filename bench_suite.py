@@ -340,6 +340,10 @@ def _single(argv):
         python bench_suite.py gemm A_BITS W_BITS SIZE
         python bench_suite.py conv BITS N C HW O KSIZE STRIDE
         python bench_suite.py fc A_BITS W_BITS M N K
+        python bench_suite.py encode BITS ROWS K            (row encoder, four inputs in rotation)
+        python bench_suite.py nchw BITS N C HW              (NCHW encoder)
+        python bench_suite.py absmax ROWS K
+        python bench_suite.py i8 SIZE                       (context: own tensor-core kernel, signed form)
     Prints the CUDA-event time of the last 10 launches."""
     dev = torch.device("cuda:0")
     torch.cuda.set_device(0)
@@ -374,6 +378,42 @@ def _single(argv):
         cf = torch.empty((m, n), dtype=torch.float32, device=dev)
         fn = lambda: mpq.gemm(ap, ab, wp, wb, m, n, k, None, cf, sa, sw, mpq.SCALE_PER_ROW)
         popcs = float(ab * wb) * m * n * (k // 32)
+    elif argv[0] in ("encode", "absmax"):
+        bits = int(argv[1]) if argv[0] == "encode" else 0
+        rows, k = (int(a) for a in argv[-2:])
+        xs = [torch.randn(rows, k, device=dev) for _ in range(4)]
+        sa = mpq.absmax(xs[0])
+        planes = torch.empty((max(bits, 1), rows, mpq.row_words(k)), dtype=torch.int32, device=dev)
+        i = [0]
+
+        def fn():
+            if bits:
+                mpq.encode(xs[i[0] % 4], sa, bits, out=planes)
+            else:
+                mpq.absmax(xs[i[0] % 4], out=sa)
+            i[0] += 1
+        popcs = 0.0
+        print("bytes per launch: %.0f" % (rows * k * (4 + bits / 8.0)))
+    elif argv[0] == "nchw":
+        bits, N, C, HW = (int(a) for a in argv[1:5])
+        xs = [torch.randn(N, C, HW, HW, device=dev).relu_() for _ in range(2)]
+        sa = mpq.absmax(xs[0], 0, mpq.ACT_HRELU)
+        planes = torch.empty((bits, N, HW, HW, C // 32), dtype=torch.int32, device=dev)
+        i = [0]
+
+        def fn():
+            mpq.encode_nchw(xs[i[0] % 2], sa, bits, mpq.ACT_HRELU, out=planes)
+            i[0] += 1
+        popcs = 0.0
+        print("bytes per launch: %.0f" % (xs[0].numel() * (4 + bits / 8.0)))
+    elif argv[0] == "i8":
+        size = int(argv[1])
+        qa = torch.randint(-3, 4, (size, size), dtype=torch.int8, device=dev)
+        qb = torch.randint(-3, 4, (size, size), dtype=torch.int8, device=dev)
+        co = torch.empty((size, size), dtype=torch.int32, device=dev)
+        err = torch.zeros(1, dtype=torch.int32, device=dev)
+        fn = lambda: context.i8_gemm(qa, qb, co, err)
+        popcs = 0.0
     else:
         raise SystemExit(_single.__doc__)
     ms = _events_ms(fn, 10, 4)
