@@ -165,6 +165,13 @@ def run_suite(dev: torch.device, hbm_gbs: float, path=None):
     rec["weight_encode"] = {"us": ms_we * 1e3, "gb_s": by / (ms_we * 1e-3) / 1e9,
                             "frac_of_hbm": by / (ms_we * 1e-3) / 1e9 / hbm_gbs}
     enc["rows_4096x9216_b2_per_row_scale"] = rec["weight_encode"]
+    # range + encode of the same weights in one pass over memory (mpq_encode_ranged) against the two-pass route
+    ms_two = _graph_ms(lambda: (mpq.absmax(w, mpq.SCALE_PER_ROW, out=sw), mpq.encode(w, sw, 2, mpq.SCALE_PER_ROW, out=wp)))
+    ms_one = _graph_ms(lambda: mpq.lib().mpq_encode_ranged(w.data_ptr(), n, k, k, mpq.ACT_HTANH, 2, sw.data_ptr(), wp.data_ptr(),
+                                                           torch.cuda.current_stream().cuda_stream))
+    enc["rows_4096x9216_b2_range_and_encode_one_pass"] = {"us": ms_one * 1e3, "gb_s": by / (ms_one * 1e-3) / 1e9,
+                                                          "frac_of_hbm": by / (ms_one * 1e-3) / 1e9 / hbm_gbs,
+                                                          "two_pass_us": ms_two * 1e3}
     out["fc_w2a2_64x4096x9216"] = rec
     del w, w2
 

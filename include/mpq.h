@@ -89,6 +89,15 @@ int mpq_encode(const float* x, int64_t rows, int64_t k, int64_t ldx,
                const float* scale, int mode, int act, int bits,
                uint32_t* planes, void* stream);
 
+/* Range and Encoder of a matrix with ONE RANGE PER ROW in a single pass over memory (weights with a
+ * range per output channel, encoded once when a layer is prepared): scale_out[r] = max |x[r][.]|
+ * (HTanh) or max of max(x, 0) (HReLU), NaNs ignored, exactly as mpq_absmax gives it, and planes as
+ * mpq_encode gives them with those ranges.  Rows of up to 49152 elements whose starts are 16-byte
+ * aligned are staged in shared memory and read from memory once; other shapes run mpq_absmax and
+ * mpq_encode one after the other (same results). */
+int mpq_encode_ranged(const float* x, int64_t rows, int64_t k, int64_t ldx, int act, int bits,
+                      float* scale_out, uint32_t* planes, void* stream);
+
 /* The same call with the form of the Encoder selectable (Section 3.2 "M-bit Encoding Functions").
  * MPQ_ENC_LEVELS is mpq_encode.  MPQ_ENC_TRIG evaluates the paper's periodic encoders literally:
  * with y = x/s limited by `act` to [-1,1] (HTanh) or [0,1] (HReLU) and L = 2^bits - 1,

@@ -49,6 +49,7 @@ def lib() -> ctypes.CDLL:
         L.mpq_absmax.argtypes = [P, i64, i64, i64, i32, i32, P, P]
         L.mpq_encode.argtypes = [P, i64, i64, i64, P, i32, i32, i32, P, P]
         L.mpq_encode_with.argtypes = [i32, P, i64, i64, i64, P, i32, i32, i32, P, P]
+        L.mpq_encode_ranged.argtypes = [P, i64, i64, i64, i32, i32, P, P, P]
         L.mpq_encode_nchw.argtypes = [P, i32, i32, i32, i32, P, i32, i32, P, P]
         L.mpq_encode_oihw.argtypes = [P, i32, i32, i32, i32, P, i32, i32, P, P, P]
         L.mpq_gemm.argtypes = [P, i32, P, i32, i64, i64, i64, P, P, i64, P, P, i32, P]
@@ -82,7 +83,7 @@ def lib() -> ctypes.CDLL:
         L.mpq_measure_b1_mma_peak.restype = i32
         for name in ("mpq_absmax", "mpq_encode", "mpq_encode_nchw", "mpq_encode_oihw", "mpq_gemm", "mpq_conv",
                      "mpq_add_relu", "mpq_stem_conv7x7", "mpq_maxpool3x3s2", "mpq_conv_fused", "mpq_zero", "mpq_linear", "mpq_linear_static", "mpq_linear_host", "mpq_measure_popc_peak",
-                     "mpq_encode_with", "mpq_gemm_fused", "mpq_conv_encoded", "mpq_linear_host_prepared"):
+                     "mpq_encode_with", "mpq_encode_ranged", "mpq_gemm_fused", "mpq_conv_encoded", "mpq_linear_host_prepared"):
             getattr(L, name).restype = i32
         _lib = L
     return _lib
@@ -142,6 +143,16 @@ def encode(x: torch.Tensor, scale: torch.Tensor, bits: int, mode: int = SCALE_PE
     _check(lib().mpq_encode(_ptr(x, torch.float32), rows, k, k, _ptr(scale, torch.float32), mode, act, bits,
                             _ptr(out, torch.int32), _stream()), "mpq_encode")
     return out
+
+
+def encode_ranged(x: torch.Tensor, bits: int, act: int = ACT_HTANH):
+    """Per-row ranges and planes of [rows x k] in one pass over memory: returns (scale [rows], planes)."""
+    rows, k = x.shape
+    scale = torch.empty(rows, dtype=torch.float32, device=x.device)
+    planes = torch.empty((bits, rows, row_words(k)), dtype=torch.int32, device=x.device)
+    _check(lib().mpq_encode_ranged(_ptr(x, torch.float32), rows, k, k, act, bits, _ptr(scale, torch.float32),
+                                   _ptr(planes, torch.int32), _stream()), "mpq_encode_ranged")
+    return scale, planes
 
 
 def encode_with(encoder: int, x: torch.Tensor, scale: torch.Tensor, bits: int, mode: int = SCALE_PER_TENSOR,

@@ -146,6 +146,54 @@ struct LaneBytes {
     }
 };
 
+// The 32 staged elements of one lane (eight consecutive 16-byte chunks at lane_row) -> its BITS plane
+// words: quantizer on the floating-point pipe, builder by code width, and the plain quantizer again
+// for a lane that met a NaN under HTanh or a range whose inverse is 0 or infinite.
+template <int BITS, int ACT>
+__device__ __forceinline__ void staged_lane_words(const float* lane_row, float inv, uint32_t two, uint32_t (&word)[BITS]) {
+    constexpr int H = 1 << (BITS - 1);
+    const float half_L = 0.5f * (float)((1 << BITS) - 1);
+    const float lo = (float)(-H), hi = (float)H - 0.5f;
+    const float4* own = reinterpret_cast<const float4*>(lane_row);
+    float probe = 0.0f;                                 // turns NaN if any element is NaN
+    if constexpr (BITS >= kByteBuilderFromBits) {
+        LaneBytes<BITS, ACT> lb;
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+            const float4 v = own[c];
+            if (ACT == MPQ_ACT_HTANH) probe = fmaf(v.x, v.y, fmaf(v.z, v.w, probe));
+            lb.set(4 * c + 0, level_fraction<BITS, ACT>(v.x, inv, half_L));
+            lb.set(4 * c + 1, level_fraction<BITS, ACT>(v.y, inv, half_L));
+            lb.set(4 * c + 2, level_fraction<BITS, ACT>(v.z, inv, half_L));
+            lb.set(4 * c + 3, level_fraction<BITS, ACT>(v.w, inv, half_L));
+        }
+        lb.words(word);
+    } else {
+        LaneWords<BITS, ACT> lw;
+        lw.clear();
+#pragma unroll
+        for (int c = 7; c >= 0; --c) {
+            const float4 v = own[c];
+            if (ACT == MPQ_ACT_HTANH) probe = fmaf(v.x, v.y, fmaf(v.z, v.w, probe));
+            lw.push(level_fraction<BITS, ACT>(v.w, inv, half_L), two);
+            lw.push(level_fraction<BITS, ACT>(v.z, inv, half_L), two);
+            lw.push(level_fraction<BITS, ACT>(v.y, inv, half_L), two);
+            lw.push(level_fraction<BITS, ACT>(v.x, inv, half_L), two);
+        }
+#pragma unroll
+        for (int p = 0; p < BITS; ++p) word[p] = lw.word(p);
+    }
+    if (ACT == MPQ_ACT_HTANH && (probe != probe || inv == 0.0f || inv == __int_as_float(0x7f800000))) {
+#pragma unroll
+        for (int p = 0; p < BITS; ++p) word[p] = 0u;
+        for (int t = 0; t < 32; ++t) {
+            const uint32_t u = (uint32_t)level_index<ACT>(lane_row[t], inv, half_L, lo, hi, H);
+#pragma unroll
+            for (int p = 0; p < BITS; ++p) word[p] |= ((u >> p) & 1u) << t;
+        }
+    }
+}
+
 template <int BITS, int ACT>
 __global__ void __launch_bounds__(kEncodeThreads)
 encode_rows_kernel(const float* __restrict__ x, int64_t rows, int64_t k, int64_t ldx,
@@ -178,45 +226,8 @@ encode_rows_kernel(const float* __restrict__ x, int64_t rows, int64_t k, int64_t
         }
         copy_async_wait_all();
         __syncwarp();
-        const float4* own = reinterpret_cast<const float4*>(mine + lane * kStageRow);
-        float probe = 0.0f;                                 // turns NaN if any element is NaN
         uint32_t word[BITS];
-        if constexpr (BITS >= kByteBuilderFromBits) {
-            LaneBytes<BITS, ACT> lb;
-#pragma unroll
-            for (int c = 0; c < 8; ++c) {
-                const float4 v = own[c];
-                if (ACT == MPQ_ACT_HTANH) probe = fmaf(v.x, v.y, fmaf(v.z, v.w, probe));
-                lb.set(4 * c + 0, level_fraction<BITS, ACT>(v.x, inv, half_L));
-                lb.set(4 * c + 1, level_fraction<BITS, ACT>(v.y, inv, half_L));
-                lb.set(4 * c + 2, level_fraction<BITS, ACT>(v.z, inv, half_L));
-                lb.set(4 * c + 3, level_fraction<BITS, ACT>(v.w, inv, half_L));
-            }
-            lb.words(word);
-        } else {
-            LaneWords<BITS, ACT> lw;
-            lw.clear();
-#pragma unroll
-            for (int c = 7; c >= 0; --c) {
-                const float4 v = own[c];
-                if (ACT == MPQ_ACT_HTANH) probe = fmaf(v.x, v.y, fmaf(v.z, v.w, probe));
-                lw.push(level_fraction<BITS, ACT>(v.w, inv, half_L), two);
-                lw.push(level_fraction<BITS, ACT>(v.z, inv, half_L), two);
-                lw.push(level_fraction<BITS, ACT>(v.y, inv, half_L), two);
-                lw.push(level_fraction<BITS, ACT>(v.x, inv, half_L), two);
-            }
-#pragma unroll
-            for (int p = 0; p < BITS; ++p) word[p] = lw.word(p);
-        }
-        if (ACT == MPQ_ACT_HTANH && (probe != probe || inv == 0.0f || inv == __int_as_float(0x7f800000))) {
-#pragma unroll
-            for (int p = 0; p < BITS; ++p) word[p] = 0u;
-            for (int t = 0; t < 32; ++t) {
-                const uint32_t u = (uint32_t)level_index<ACT>(mine[lane * kStageRow + t], inv, half_L, lo, hi, H);
-#pragma unroll
-                for (int p = 0; p < BITS; ++p) word[p] |= ((u >> p) & 1u) << t;
-            }
-        }
+        staged_lane_words<BITS, ACT>(mine + lane * kStageRow, inv, two, word);
         uint32_t* dst = planes + row * rw + seg * 32 + lane;
         const int64_t plane_stride = rows * rw;
 #pragma unroll
@@ -251,6 +262,83 @@ encode_rows_kernel(const float* __restrict__ x, int64_t rows, int64_t k, int64_t
     if (word_idx < rw) {
 #pragma unroll
         for (int p = 0; p < BITS; ++p) planes[((int64_t)p * rows + row) * rw + word_idx] = mine[p];
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// Per-row range AND encode in one pass over HBM (weights with one range per output channel): one
+// CTA stages a whole row in shared memory (the same 32 x 36 layout per 1024-element segment),
+// takes the row's maximum there, publishes it, and encodes the segments from the staged copy, so
+// the row is read from HBM once instead of twice.  Rows of up to kRangedMaxK elements.
+// ------------------------------------------------------------------------------------------
+constexpr int64_t kRangedMaxK = 48 * 1024;                      // 48 segments x 4608 bytes = 216 KiB staged
+
+template <int BITS, int ACT>
+__global__ void __launch_bounds__(kEncodeThreads)
+encode_rows_ranged_kernel(const float* __restrict__ x, int64_t rows, int64_t k, int64_t ldx,
+                          float* __restrict__ scale_out, uint32_t* __restrict__ planes, int64_t rw, uint32_t two) {
+    extern __shared__ __align__(16) float staged[];             // [segments][32 * kStageRow]
+    __shared__ float warp_max[kEncodeThreads / 32];
+    chain_entry();
+    const int64_t row = blockIdx.x;
+    const float* xr = x + row * ldx;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int64_t full_chunks = k / 4;                          // 16-byte chunks that lie wholly inside the row
+    const int segs = (int)ceil_div(k, 1024);
+    // stage: chunk c -> segment c / 256, row (c % 256) / 8 of the segment, 16-byte slot (c % 8)
+    for (int64_t c = tid; c < full_chunks; c += kEncodeThreads) {
+        const int cc = (int)(c & 255);
+        copy_async_16(staged + (c >> 8) * (32 * kStageRow) + (cc >> 3) * kStageRow + (cc & 7) * 4, xr + c * 4);
+    }
+    // the ragged end of the row and the rest of its last segment: plain stores (zeros past the end)
+    for (int64_t e = full_chunks * 4 + tid; e < (int64_t)segs * 1024; e += kEncodeThreads) {
+        const int ee = (int)(e & 1023);
+        staged[(e >> 10) * (32 * kStageRow) + (ee >> 5) * kStageRow + (ee & 31)] = e < k ? __ldg(xr + e) : 0.0f;
+    }
+    copy_async_wait_all();
+    __syncthreads();
+    // range of the row
+    float m = 0.0f;
+    for (int64_t c = tid; c < (int64_t)segs * 256; c += kEncodeThreads) {
+        const int cc = (int)(c & 255);
+        const float4 v = *reinterpret_cast<const float4*>(staged + (c >> 8) * (32 * kStageRow) + (cc >> 3) * kStageRow + (cc & 7) * 4);
+        if (ACT == MPQ_ACT_HRELU) m = fmaxf(m, fmaxf(fmaxf(v.x, v.y), fmaxf(v.z, v.w)));
+        else m = fmaxf(m, fmaxf(fmaxf(fabsf(v.x), fabsf(v.y)), fmaxf(fabsf(v.z), fabsf(v.w))));
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+    if (lane == 0) warp_max[warp] = m;
+    __syncthreads();
+    m = warp_max[0];
+#pragma unroll
+    for (int w = 1; w < kEncodeThreads / 32; ++w) m = fmaxf(m, warp_max[w]);
+    if (tid == 0) scale_out[row] = m;
+    const float inv = inverse_scale(m);
+    // encode: warp w takes segments w, w + 8, ...; lane L owns word L of every plane of the segment
+    constexpr int H = 1 << (BITS - 1);
+    const float half_L = 0.5f * (float)((1 << BITS) - 1);
+    const float lo = (float)(-H), hi = (float)H - 0.5f;
+    const int64_t plane_stride = rows * rw;
+    for (int seg = warp; seg < segs; seg += kEncodeThreads / 32) {
+        const float* lane_row = staged + (size_t)seg * (32 * kStageRow) + lane * kStageRow;
+        const int64_t e0 = (int64_t)seg * 1024 + 32 * lane;    // first element of this lane's word
+        uint32_t word[BITS];
+        if (e0 + 32 <= k) {
+            staged_lane_words<BITS, ACT>(lane_row, inv, two, word);
+        } else {                                                // the word holding the end of the row, and pad words
+#pragma unroll
+            for (int p = 0; p < BITS; ++p) word[p] = 0u;
+            for (int t = 0; t < 32 && e0 + t < k; ++t) {
+                const uint32_t u = (uint32_t)level_index<ACT>(lane_row[t], inv, half_L, lo, hi, H);
+#pragma unroll
+                for (int p = 0; p < BITS; ++p) word[p] |= ((u >> p) & 1u) << t;
+            }
+        }
+        const int64_t word_idx = (int64_t)seg * 32 + lane;
+        if (word_idx < rw) {
+#pragma unroll
+            for (int p = 0; p < BITS; ++p) planes[p * plane_stride + row * rw + word_idx] = word[p];
+        }
     }
 }
 
@@ -432,6 +520,20 @@ struct EncodeNchwLauncher {
     }
 };
 
+template <int BITS, int ACT>
+struct EncodeRangedLauncher {
+    static int run(const float* x, int64_t rows, int64_t k, int64_t ldx, float* scale_out, uint32_t* planes, cudaStream_t st) {
+        const int64_t rw = row_words(k);
+        const size_t smem = (size_t)ceil_div(k, 1024) * 32 * kStageRow * sizeof(float);
+        auto kern = encode_rows_ranged_kernel<BITS, ACT>;
+        static PerDeviceOnce configured;
+        if (configured.raise_smem_limit(kern, (size_t)ceil_div(kRangedMaxK, 1024) * 32 * kStageRow * sizeof(float)) != MPQ_OK)
+            return MPQ_ERR_CUDA;
+        if (rows > 0x7fffffffLL) return MPQ_ERR_BAD_SHAPE;
+        return launch_chained(kern, (unsigned)rows, kEncodeThreads, smem, st, x, rows, k, ldx, scale_out, planes, rw, 2u);
+    }
+};
+
 }  // namespace mpq
 
 using namespace mpq;
@@ -468,6 +570,20 @@ extern "C" int mpq_encode(const float* x, int64_t rows, int64_t k, int64_t ldx,
     if (!aligned16(planes)) return MPQ_ERR_ALIGN;
     return dispatch_bits_act<EncodeRowsLauncher>(bits, act, x, rows, k, ldx, scale,
                                                  (int)(mode == MPQ_SCALE_PER_ROW), planes, (cudaStream_t)stream);
+}
+
+extern "C" int mpq_encode_ranged(const float* x, int64_t rows, int64_t k, int64_t ldx, int act, int bits,
+                                 float* scale_out, uint32_t* planes, void* stream) {
+    if (!x || !scale_out || !planes) return MPQ_ERR_NULL;
+    if (rows <= 0 || k <= 0 || ldx < k) return MPQ_ERR_BAD_SHAPE;
+    if (!bits_ok(bits) || (act != MPQ_ACT_HTANH && act != MPQ_ACT_HRELU)) return MPQ_ERR_UNSUPPORTED;
+    if (!aligned16(planes)) return MPQ_ERR_ALIGN;
+    // one pass when a row fits the staging buffer and its start is 16-byte aligned; else range, then encode
+    if (k <= kRangedMaxK && aligned16(x) && (ldx % 4 == 0 || rows == 1))
+        return dispatch_bits_act<EncodeRangedLauncher>(bits, act, x, rows, k, ldx, scale_out, planes, (cudaStream_t)stream);
+    const int rc = mpq_absmax(x, rows, k, ldx, MPQ_SCALE_PER_ROW, act, scale_out, stream);
+    if (rc != MPQ_OK) return rc;
+    return mpq_encode(x, rows, k, ldx, scale_out, MPQ_SCALE_PER_ROW, act, bits, planes, stream);
 }
 
 static bool conv_channels_ok(int C) { return C == 32 || C == 64 || (C > 0 && C % 128 == 0); }

@@ -241,3 +241,30 @@ def test_linear_host_prepared(mpq, cuda, m, n, k, per_row):
     rc = mpq.lib().mpq_linear_host_prepared(xh.data_ptr(), wp.data_ptr(), sw.data_ptr(), m, n, k, 3, 4, 1, int(per_row),
                                             oi.data_ptr(), None, small.data_ptr(), small.numel(), None)
     assert rc == 7
+
+
+# -------------------------------------------------------------- per-row range + encode in one pass
+@pytest.mark.parametrize("bits", [1, 2, 4, 8])
+@pytest.mark.parametrize("shape", [(1, 1), (5, 33), (7, 1000), (3, 1024), (6, 2500), (4, 9216), (2, 49152), (2, 50000)])
+def test_encode_ranged_equals_range_then_encode(mpq, cuda, bits, shape):
+    """One pass over memory gives the oracle's per-row ranges and the oracle's codes under those ranges
+    (NaN ignored by the range and sent to the level above zero; ties, infinities beyond the range; rows
+    longer than the staging buffer take the two-pass route with the same results)."""
+    rng = np.random.default_rng(bits * 1000 + shape[1])
+    x = (rng.standard_normal(shape) * rng.uniform(0.01, 3.0, size=(shape[0], 1))).astype(np.float32)
+    x.flat[::9] = 0.0
+    if shape[1] > 40:
+        x[0, 5] = np.nan
+        x[-1, 7] = -1e30
+    xd = _dev(x, cuda)
+    for act in (mpq.ACT_HTANH, mpq.ACT_HRELU):
+        s_ref = oracle.absmax(x, True, act)
+        scale, planes = mpq.encode_ranged(xd, bits, act)
+        assert np.array_equal(scale.cpu().numpy(), s_ref)
+        u = unpack_planes(planes.cpu().numpy(), shape[1])
+        assert np.array_equal(u, oracle.levels(oracle.quantize(x, s_ref, bits, per_row=True, act=act), bits))
+    # an all-zero row has range 0: every code is the level above zero
+    z = torch.zeros((2, 300), dtype=torch.float32, device=cuda)
+    scale, planes = mpq.encode_ranged(z, bits)
+    assert float(scale.abs().max()) == 0.0
+    assert np.all(unpack_planes(planes.cpu().numpy(), 300) == 2 ** (bits - 1))
