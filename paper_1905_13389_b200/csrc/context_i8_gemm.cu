@@ -11,11 +11,11 @@
 //         sum q_a q_b = 4 sum u_a u_b - 2 L_b sum u_a - 2 L_a sum u_b + k L_a L_b,
 //     with the row sums of u supplied by row_sums_u8 below.
 //
-// Structure: one CTA of 128 threads per 128 x 128 output tile.  Warp 0 (one lane) streams 128-byte
+// Structure: one CTA of 128 threads per 128 x 256 output tile.  Warp 0 (one lane) streams 128-byte
 // wide k-blocks of both operands through a 4-stage shared-memory ring with TMA (tiled 2-D loads,
 // 128-byte swizzle, no multicast; the tensor maps cover this GPU's own memory), warp 1 (one lane)
-// issues tcgen05.mma kind::i8 (M = 128, N = 128, K = 32 per instruction, four per k-block) into a
-// 128-column TMEM accumulator and releases ring slots with tcgen05.commit; all four warps read the
+// issues tcgen05.mma kind::i8 (M = 128, N = 256, K = 32 per instruction, four per k-block) into a
+// 256-column TMEM accumulator and releases ring slots with tcgen05.commit; all four warps read the
 // accumulator back with tcgen05.ld (warp w owns TMEM lanes 32 w .. 32 w + 31 = output rows) and
 // store 128-byte row pieces.  Every wait on an mbarrier is bounded: after kSpinLimit polls the CTA
 // raises *error_flag, stops issuing work, waits (bounded again) for its copies in flight, frees its
@@ -26,10 +26,10 @@
 
 namespace {
 
-constexpr int BM = 128, BN = 128, BK = 128;        // BK in bytes = elements
+constexpr int BM = 128, BN = 256, BK = 128;        // BK in bytes = elements
 constexpr int STAGES = 4;
-constexpr int STAGE_BYTES = (BM + BN) * BK;          // 32 KiB
-constexpr int TMEM_COLS = 128;
+constexpr int STAGE_BYTES = (BM + BN) * BK;          // 48 KiB
+constexpr int TMEM_COLS = BN;                         // one 32-bit column per output column
 constexpr uint32_t kSpinLimit = 1u << 20;
 
 __device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -71,7 +71,7 @@ __device__ __forceinline__ uint64_t umma_desc_k_major_sw128(uint32_t saddr) {
     return d;
 }
 // Instruction descriptor of kind::i8: int32 accumulator, both operands signed or both unsigned
-// 8-bit, both K-major, N = 128, M = 128.
+// 8-bit, both K-major, N = BN, M = BM.
 __host__ __device__ constexpr uint32_t umma_idesc_i8(bool is_signed) {
     return (2u << 4) | ((is_signed ? 1u : 0u) << 7) | ((is_signed ? 1u : 0u) << 10) | ((uint32_t)(BN >> 3) << 17) |
            ((uint32_t)(BM >> 4) << 24);
@@ -169,8 +169,11 @@ i8_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     if (ok) {
         const int row = m0 + warp * 32 + lane;
-        const int64_t row_term = g.is_unsigned ? (int64_t)2 * g.Lb * g.sums_a[row] : 0;
-        const int64_t constant = g.is_unsigned ? g.k * g.La * g.Lb : 0;
+        // Eq. 17 summed over k: 4 sum u_a u_b - 2 L_b sum u_a - 2 L_a sum u_b + k L_a L_b.  The result fits
+        // int32 (it is the layer's accumulator), so the terms are combined modulo 2^32.
+        const uint32_t row_term = g.is_unsigned ? 2u * (uint32_t)g.Lb * (uint32_t)g.sums_a[row] : 0u;
+        const uint32_t constant = g.is_unsigned ? (uint32_t)g.k * (uint32_t)g.La * (uint32_t)g.Lb : 0u;
+        const uint32_t col_factor = 2u * (uint32_t)g.La;
 #pragma unroll 1
         for (int chunk = 0; chunk < BN / 32; ++chunk) {
             uint32_t v[32];
@@ -185,17 +188,18 @@ i8_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                          : "r"(taddr) : "memory");
             asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
             int32_t* dst = g.c + (int64_t)row * g.n + n0 + chunk * 32;
+            const int4* col_sums = g.is_unsigned ? reinterpret_cast<const int4*>(g.sums_b + n0 + chunk * 32) : nullptr;
 #pragma unroll
             for (int j = 0; j < 32; j += 4) {
-                int32_t o[4];
-#pragma unroll
-                for (int t = 0; t < 4; ++t) {
-                    int64_t val = (int32_t)v[j + t];
-                    if (g.is_unsigned)        // Eq. 17 summed over k: 4 sum u_a u_b - 2 L_b sum u_a - 2 L_a sum u_b + k L_a L_b
-                        val = 4 * val - row_term - (int64_t)2 * g.La * g.sums_b[n0 + chunk * 32 + j + t] + constant;
-                    o[t] = (int32_t)val;
+                uint32_t o[4] = {v[j], v[j + 1], v[j + 2], v[j + 3]};
+                if (g.is_unsigned) {
+                    const int4 sb = __ldg(col_sums + j / 4);
+                    o[0] = 4u * o[0] - row_term - col_factor * (uint32_t)sb.x + constant;
+                    o[1] = 4u * o[1] - row_term - col_factor * (uint32_t)sb.y + constant;
+                    o[2] = 4u * o[2] - row_term - col_factor * (uint32_t)sb.z + constant;
+                    o[3] = 4u * o[3] - row_term - col_factor * (uint32_t)sb.w + constant;
                 }
-                *reinterpret_cast<int4*>(dst + j) = make_int4(o[0], o[1], o[2], o[3]);
+                *reinterpret_cast<int4*>(dst + j) = make_int4((int)o[0], (int)o[1], (int)o[2], (int)o[3]);
             }
         }
     }
@@ -222,11 +226,11 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-// [rows][k] bytes, k contiguous; box = 128 rows x 128 bytes, 128-byte swizzle.
-int make_map(EncodeTiledFn encode, CUtensorMap* map, const void* base, int64_t rows, int64_t k) {
+// [rows][k] bytes, k contiguous; box = box_rows rows x 128 bytes, 128-byte swizzle.
+int make_map(EncodeTiledFn encode, CUtensorMap* map, const void* base, int64_t rows, int64_t k, int box_rows) {
     const cuuint64_t dims[2] = {(cuuint64_t)k, (cuuint64_t)rows};
     const cuuint64_t strides[1] = {(cuuint64_t)k};
-    const cuuint32_t box[2] = {BK, BM};
+    const cuuint32_t box[2] = {BK, (cuuint32_t)box_rows};
     const cuuint32_t elem[2] = {1, 1};
     return encode(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, elem,
                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
@@ -235,8 +239,8 @@ int make_map(EncodeTiledFn encode, CUtensorMap* map, const void* base, int64_t r
 
 }  // namespace
 
-// Status: 0 ok, 1 null pointer, 2 bad shape (m, n, k must be multiples of 128; k < 2^24), 5 alignment
-// (operands 16-byte aligned), 6 CUDA / driver error.  *error_flag (device int, zeroed by the caller)
+// Status: 0 ok, 1 null pointer, 2 bad shape (m, k multiples of 128, n a multiple of 256; k < 2^24), 5 alignment
+// (operands, output and sums_b 16-byte aligned), 6 CUDA / driver error.  *error_flag (device int, zeroed by the caller)
 // is raised by a CTA whose bounded wait ran out.
 extern "C" int mpqctx_i8_gemm(const void* a, const void* b, int64_t m, int64_t n, int64_t k, int32_t* c,
                               int is_unsigned, const int32_t* sums_a, const int32_t* sums_b, int La, int Lb,
@@ -244,6 +248,7 @@ extern "C" int mpqctx_i8_gemm(const void* a, const void* b, int64_t m, int64_t n
     if (!a || !b || !c || !error_flag || (is_unsigned && (!sums_a || !sums_b))) return 1;
     if (m <= 0 || n <= 0 || k <= 0 || m % BM || n % BN || k % BK || k >= (1 << 24) || m / BM > 65535) return 2;
     if ((reinterpret_cast<uintptr_t>(a) | reinterpret_cast<uintptr_t>(b) | reinterpret_cast<uintptr_t>(c)) & 15u) return 5;
+    if (is_unsigned && (reinterpret_cast<uintptr_t>(sums_b) & 15u)) return 5;
     static EncodeTiledFn encode = nullptr;
     if (!encode) {
         void* fn = nullptr;
@@ -252,7 +257,7 @@ extern "C" int mpqctx_i8_gemm(const void* a, const void* b, int64_t m, int64_t n
         encode = reinterpret_cast<EncodeTiledFn>(fn);
     }
     CUtensorMap map_a, map_b;
-    if (make_map(encode, &map_a, a, m, k) || make_map(encode, &map_b, b, n, k)) return 6;
+    if (make_map(encode, &map_a, a, m, k, BM) || make_map(encode, &map_b, b, n, k, BN)) return 6;
     const size_t smem = (size_t)STAGES * STAGE_BYTES + 1024;
     static bool configured = false;
     if (!configured) {

@@ -12,7 +12,7 @@ from paper_1905_13389_b200 import context, inputs
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("m,n,k", [(128, 128, 128), (256, 384, 1024), (512, 256, 4096)])
+@pytest.mark.parametrize("m,n,k", [(128, 256, 128), (256, 768, 1024), (512, 256, 4096)])
 @pytest.mark.parametrize("a_bits,w_bits", [(2, 2), (4, 7), (7, 3)])
 def test_signed_form_equals_the_oracle(mpq, cuda, m, n, k, a_bits, w_bits):
     x = inputs.uniform_levels(15, a_bits, (m, k), a_bits)
@@ -37,7 +37,7 @@ def test_signed_form_equals_the_oracle(mpq, cuda, m, n, k, a_bits, w_bits):
     assert torch.equal(ci, out)
 
 
-@pytest.mark.parametrize("m,n,k", [(128, 256, 512), (256, 128, 4096)])
+@pytest.mark.parametrize("m,n,k", [(128, 256, 512), (256, 512, 4096)])
 def test_unsigned_form_with_eq17_correction_equals_the_oracle(mpq, cuda, m, n, k):
     """8-bit codes: |q| reaches 255, so the operands are the level indices u and the store applies
     4 sum u_a u_b - 2 L_b sum u_a - 2 L_a sum u_b + k L_a L_b."""
@@ -59,11 +59,12 @@ def test_unsigned_form_with_eq17_correction_equals_the_oracle(mpq, cuda, m, n, k
 
 
 def test_shapes_outside_the_tile_grid_are_refused(cuda):
-    a = torch.zeros((128, 128), dtype=torch.int8, device=cuda)
-    out = torch.zeros((128, 128), dtype=torch.int32, device=cuda)
+    a = torch.zeros((256, 128), dtype=torch.int8, device=cuda)
+    out = torch.zeros((128, 256), dtype=torch.int32, device=cuda)
     err = torch.zeros(1, dtype=torch.int32, device=cuda)
     L = context.lib()
-    assert L.mpqctx_i8_gemm(a.data_ptr(), a.data_ptr(), 100, 128, 128, out.data_ptr(), 0, None, None, 0, 0, err.data_ptr(), None) == 2
-    assert L.mpqctx_i8_gemm(a.data_ptr(), a.data_ptr(), 128, 128, 96, out.data_ptr(), 0, None, None, 0, 0, err.data_ptr(), None) == 2
-    assert L.mpqctx_i8_gemm(None, a.data_ptr(), 128, 128, 128, out.data_ptr(), 0, None, None, 0, 0, err.data_ptr(), None) == 1
-    assert L.mpqctx_i8_gemm(a.data_ptr(), a.data_ptr(), 128, 128, 128, out.data_ptr(), 1, None, None, 3, 3, err.data_ptr(), None) == 1
+    assert L.mpqctx_i8_gemm(a.data_ptr(), a.data_ptr(), 100, 256, 128, out.data_ptr(), 0, None, None, 0, 0, err.data_ptr(), None) == 2
+    assert L.mpqctx_i8_gemm(a.data_ptr(), a.data_ptr(), 128, 128, 128, out.data_ptr(), 0, None, None, 0, 0, err.data_ptr(), None) == 2
+    assert L.mpqctx_i8_gemm(a.data_ptr(), a.data_ptr(), 128, 256, 96, out.data_ptr(), 0, None, None, 0, 0, err.data_ptr(), None) == 2
+    assert L.mpqctx_i8_gemm(None, a.data_ptr(), 128, 256, 128, out.data_ptr(), 0, None, None, 0, 0, err.data_ptr(), None) == 1
+    assert L.mpqctx_i8_gemm(a.data_ptr(), a.data_ptr(), 128, 256, 128, out.data_ptr(), 1, None, None, 3, 3, err.data_ptr(), None) == 1

@@ -105,3 +105,82 @@ def test_two_streams_run_independent_layers(mpq, cuda):
     for c in cases:
         assert np.array_equal(c["oi"].cpu().numpy(), c["acc"])
         assert rel_close(c["of"].cpu().numpy(), c["out"])
+
+
+def _pack_nhwc(u, bits):
+    """Level indices [N][O][Ho][Wo] -> planes [bits][N][Ho][Wo][O/32] (test-side packer)."""
+    N, O, Ho, Wo = u.shape
+    t = u.transpose(0, 2, 3, 1).reshape(N, Ho, Wo, O // 32, 32).astype(np.uint64)
+    weights = np.uint64(1) << np.arange(32, dtype=np.uint64)
+    return np.stack([(((t >> np.uint64(p)) & np.uint64(1)) * weights).sum(axis=4).astype(np.uint32) for p in range(bits)])
+
+
+@pytest.mark.parametrize("seed", range(16))
+def test_gemm_fused_random_cases(mpq, cuda, seed):
+    """The glue in the GEMM store (bias, residual, max in any combination) on random shapes, among them
+    few-tile / long-k shapes that run with k-groups inside the CTA."""
+    rng = np.random.default_rng(3000 + seed)
+    a_bits, w_bits = int(rng.integers(1, 9)), int(rng.integers(1, 9))
+    m = int(rng.choice([1, 17, 64, 100]))
+    n = int(rng.choice([3, 100, 1000, 2500, 4096]))
+    k = int(rng.choice([129, 1024, 3000, 9216, 20000]))
+    while (2 ** a_bits - 1) * (2 ** w_bits - 1) * k >= 2 ** 31:
+        k //= 2
+    per_row = bool(rng.integers(0, 2))
+    x = inputs.uniform_levels(24, 2 * seed, (m, k), a_bits)
+    w = inputs.uniform_levels(24, 2 * seed + 1, (n, k), w_bits)
+    acc_ref, out_ref, _, _ = oracle.linear(x, w, a_bits, w_bits, w_per_row=per_row)
+    scale = float(np.abs(out_ref).max()) or 1.0
+    bias = (rng.standard_normal(n) * 0.3 * scale).astype(np.float32) if rng.integers(0, 2) else None
+    res = (rng.standard_normal((m, n)) * 0.3 * scale).astype(np.float32) if rng.integers(0, 2) else None
+    relu = bool(rng.integers(0, 2))
+    ref = oracle.epilogue(out_ref, bias, res, relu)
+    xd, wd = _dev(x, cuda), _dev(w, cuda)
+    sa_d, sw_d = mpq.absmax(xd), mpq.absmax(wd, int(per_row))
+    ap, wp = mpq.encode(xd, sa_d, a_bits), mpq.encode(wd, sw_d, w_bits, int(per_row))
+    ci = torch.full((m, n), -5, dtype=torch.int32, device=cuda)
+    cf = torch.full((m, n), float("nan"), dtype=torch.float32, device=cuda)
+    mpq.gemm_fused(ap, a_bits, wp, w_bits, m, n, k, ci, cf, sa_d, sw_d, int(per_row),
+                   None if bias is None else _dev(bias, cuda), None if res is None else _dev(res, cuda), relu)
+    key = (a_bits, w_bits, m, n, k, per_row, bias is not None, res is not None, relu)
+    assert np.array_equal(ci.cpu().numpy(), acc_ref), key
+    assert rel_close(cf.cpu().numpy(), ref), key
+
+
+@pytest.mark.parametrize("seed", range(16))
+def test_conv_encoded_random_cases(mpq, cuda, seed):
+    """The consumer's Encoder in the convolution's store on random layers: planes equal the oracle's codes
+    of the oracle's (glued) fp32 output under a range fixed beforehand."""
+    rng = np.random.default_rng(4000 + seed)
+    a_bits, w_bits, next_bits = int(rng.integers(1, 9)), int(rng.integers(1, 9)), int(rng.integers(1, 9))
+    C = int(rng.choice([32, 64, 128, 256]))
+    ksz = int(rng.choice([1, 3]))
+    stride = int(rng.choice([1, 2]))
+    pad = int(rng.integers(0, 2)) if ksz == 3 else 0
+    H, W = int(rng.integers(3, 16)), int(rng.integers(3, 16))
+    N = int(rng.choice([1, 2, 5]))
+    O = int(rng.choice([32, 64, 96, 160]))
+    if a_bits + w_bits > 12 and C > 128:
+        C = 128
+    x = inputs.uniform_levels(25, 2 * seed, (N, C, H, W), a_bits)
+    w = inputs.uniform_levels(25, 2 * seed + 1, (O, C, ksz, ksz), w_bits)
+    acc_ref, out_ref, _, _ = oracle.conv_layer(x, w, a_bits, w_bits, stride, pad, True, oracle.HTANH)
+    res = (rng.standard_normal(out_ref.shape) * 0.4 * np.abs(out_ref).max()).astype(np.float32) if rng.integers(0, 2) else None
+    relu = bool(rng.integers(0, 2))
+    act = int(rng.integers(0, 2))
+    ref = oracle.epilogue(out_ref, None, res, relu)
+    s_next = np.array([rng.uniform(0.3, 1.2) * max(float(np.abs(ref).max()), 1e-6)], np.float32)
+    want = _pack_nhwc(oracle.levels(oracle.quantize(ref, s_next, next_bits, act=act), next_bits), next_bits)
+    xd, wd = _dev(x, cuda), _dev(w, cuda)
+    sa_d, sw_d = mpq.absmax(xd), mpq.absmax(wd, mpq.SCALE_PER_ROW)
+    xp = mpq.encode_nchw(xd, sa_d, a_bits)
+    wp, taps = mpq.encode_oihw(wd, sw_d, w_bits, mpq.SCALE_PER_ROW)
+    keep = bool(rng.integers(0, 2))
+    yf = torch.full(acc_ref.shape, float("nan"), dtype=torch.float32, device=cuda) if keep else None
+    planes = mpq.conv_encoded(xp, a_bits, N, C, H, W, wp, w_bits, taps, O, ksz, ksz, stride, pad, None, yf, sa_d, sw_d,
+                              mpq.SCALE_PER_ROW, None if res is None else _dev(res, cuda), relu, None,
+                              _dev(s_next, cuda), act, next_bits)
+    key = (a_bits, w_bits, next_bits, N, C, H, W, O, ksz, stride, pad, res is not None, relu, act)
+    assert np.array_equal(planes.cpu().numpy().view(np.uint32), want), key
+    if keep:
+        assert np.array_equal(yf.cpu().numpy(), ref), key
