@@ -1,6 +1,6 @@
 // Context only -- NOT part of libmpq.so and never a backend of the library.
 //
-// What the bit-plane method costs on this chip is judged against the product of the DECODED
+// What the bit-plane method costs on this chip is measured against the product of the DECODED
 // integers on the 5th-generation tensor cores (Eq. 16-18: the layer's result is an ordinary integer
 // dot product of the odd levels q, or of the level indices u with the correction terms of Eq. 17).
 // This file is that comparison kernel, written for sm_100a: C[m][n] = sum_t A[m][t] * B[n][t] with
