@@ -115,7 +115,7 @@ def run_suite(dev: torch.device, hbm_gbs: float, path=None):
         "signed_ms": ms, "signed_tops": 2.0 * size ** 3 / (ms * 1e-3) / 1e12,
         "unsigned_eq17_ms": ms_u, "unsigned_eq17_tops": 2.0 * size ** 3 / (ms_u * 1e-3) / 1e12,
         "bounded_wait_ran_out": int(err.cpu()[0]),
-        "note": "decoded-integer product on the 5th-generation tensor cores, own kernel (128 x 256 tile, one CTA per SM, "
+        "note": "decoded-integer product on the 5th-generation tensor cores, own kernel (persistent, 128 x 256 tile, two TMEM accumulators, "
                 "no multicast); context for the bit-plane numbers, not part of the library"}
     del qa, qb, ua, ub, co
 

@@ -12,9 +12,10 @@ from paper_1905_13389_b200 import context, inputs
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("m,n,k", [(128, 256, 128), (256, 768, 1024), (512, 256, 4096)])
+@pytest.mark.parametrize("m,n,k", [(128, 256, 128), (256, 768, 1024), (512, 256, 4096), (4096, 4096, 128)])
 @pytest.mark.parametrize("a_bits,w_bits", [(2, 2), (4, 7), (7, 3)])
 def test_signed_form_equals_the_oracle(mpq, cuda, m, n, k, a_bits, w_bits):
+    """(4096 x 4096 x 128 is 512 tiles for 148 persistent CTAs: both TMEM accumulators get reused.)"""
     x = inputs.uniform_levels(15, a_bits, (m, k), a_bits)
     w = inputs.uniform_levels(15, 10 + w_bits, (n, k), w_bits)
     qa = oracle.quantize(x, 1.0, a_bits)
@@ -37,7 +38,7 @@ def test_signed_form_equals_the_oracle(mpq, cuda, m, n, k, a_bits, w_bits):
     assert torch.equal(ci, out)
 
 
-@pytest.mark.parametrize("m,n,k", [(128, 256, 512), (256, 512, 4096)])
+@pytest.mark.parametrize("m,n,k", [(128, 256, 512), (256, 512, 4096), (3072, 4096, 256)])
 def test_unsigned_form_with_eq17_correction_equals_the_oracle(mpq, cuda, m, n, k):
     """8-bit codes: |q| reaches 255, so the operands are the level indices u and the store applies
     4 sum u_a u_b - 2 L_b sum u_a - 2 L_a sum u_b + k L_a L_b."""
