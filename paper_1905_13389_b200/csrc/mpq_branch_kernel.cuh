@@ -487,9 +487,14 @@ branch_kernel(const BranchParams p) {
         }
         float seen_max = 0.0f;
         // consumer's Encoder in the store: its level indices go through a [pixel][channel] byte tile in the
-        // (drained) staging ring, then one ballot per plane packs 32 channels of a pixel into a word
+        // (drained) staging ring; one thread per pixel and 32-channel group then turns 32 bytes into plane
+        // words with an 8 x 8 bit-block transpose.  Channel c of a group sits at byte 4 (c % 8) + c / 8, so
+        // 32-bit word i of the pixel holds channels i, 8 + i, 16 + i, 24 + i: the transpose's input order
+        // (a 16-channel tile keeps channels i, 8 + i in 16-bit half i and fills half a plane word).
+        // A pixel takes BH + 4 bytes (an odd number of words: neighbouring pixels fall into distinct banks).
         const bool want_planes = p.next_planes != nullptr;
         unsigned char* code_tile = reinterpret_cast<unsigned char*>(smem);
+        constexpr int PIXEL_BYTES = BH + 4;
         float next_inv = 0.0f, next_half_L = 0.0f, next_lo = 0.0f, next_hi = 0.0f;
         int next_H = 0;
         if (want_planes) {
@@ -531,31 +536,48 @@ branch_kernel(const BranchParams p) {
                         const int u = p.next_act == MPQ_ACT_HRELU
                                           ? level_index<MPQ_ACT_HRELU>(f, next_inv, next_half_L, next_lo, next_hi, next_H)
                                           : level_index<MPQ_ACT_HTANH>(f, next_inv, next_half_L, next_lo, next_hi, next_H);
-                        code_tile[r * BH + ty + 16 * a] = (unsigned char)u;
+                        const int c = ty + 16 * a;
+                        const int at = BH >= 32 ? (c & ~31) + 4 * (c & 7) + ((c >> 3) & 3) : 2 * (c & 7) + (c >> 3);
+                        code_tile[r * PIXEL_BYTES + at] = (unsigned char)u;
                     }
                 }
             }
         }
         if (want_planes) {
             __syncthreads();
-            // (pixel, 32-channel group) pairs of the tile, one per warp and step; lane = channel
+            // (pixel, 32-channel group) pairs of the tile, one per thread
             constexpr int GROUPS = BH >= 32 ? BH / 32 : 1;
-            constexpr int LANES = BH >= 32 ? 32 : BH;          // a 16-channel tile fills half a word
-            const int lane = tid & 31, warp = tid >> 5;
             const int Ow = p.O / 32;
             const int64_t plane_words = (int64_t)p.N * hw * Ow;
-            for (int task = warp; task < BS * GROUPS; task += 8) {
+            for (int task = tid; task < BS * GROUPS; task += 256) {
                 const int r = task / GROUPS, grp = task % GROUPS;
                 const int n = row_n[r];
                 const int64_t o0 = h0 + 32 * grp;
-                const bool live = n >= 0 && o0 < p.held_rows;      // warp-uniform
-                const unsigned u = (live && lane < LANES) ? code_tile[r * BH + 32 * grp + lane] : 0u;
-                for (int q = 0; q < p.next_bits; ++q) {
-                    const unsigned word = __ballot_sync(0xffffffffu, (u >> q) & 1u);
-                    if (live && lane == q) {
-                        const int64_t at = (int64_t)q * plane_words + ((int64_t)n * hw + row_rem[r]) * Ow + o0 / 32;
-                        if (BH >= 32) p.next_planes[at] = word;
-                        else reinterpret_cast<unsigned short*>(p.next_planes)[2 * at + ((o0 >> 4) & 1)] = (unsigned short)word;
+                if (n < 0 || o0 >= p.held_rows) continue;
+                const uint32_t* mine = reinterpret_cast<const uint32_t*>(code_tile + r * PIXEL_BYTES + 32 * grp);
+                uint32_t w[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i)
+                    w[i] = BH >= 32 ? mine[i] : (mine[i >> 1] >> (16 * (i & 1))) & 0x0000FFFFu;
+#pragma unroll
+                for (int d = 1; d <= 4; d *= 2) {
+                    const uint32_t mask = d == 1 ? 0x55555555u : d == 2 ? 0x33333333u : 0x0F0F0F0Fu;
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        if ((i & d) == 0) {
+                            const uint32_t x = ((w[i] >> d) ^ w[i + d]) & mask;
+                            w[i + d] ^= x;
+                            w[i] ^= x << d;
+                        }
+                    }
+                }
+                const int64_t at0 = ((int64_t)n * hw + row_rem[r]) * Ow + o0 / 32;
+#pragma unroll
+                for (int q = 0; q < 8; ++q) {
+                    if (q < p.next_bits) {
+                        const int64_t at = (int64_t)q * plane_words + at0;
+                        if (BH >= 32) p.next_planes[at] = w[q];
+                        else reinterpret_cast<unsigned short*>(p.next_planes)[2 * at + ((o0 >> 4) & 1)] = (unsigned short)w[q];
                     }
                 }
             }
