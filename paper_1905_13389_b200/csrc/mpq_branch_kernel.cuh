@@ -58,6 +58,7 @@ struct BranchParams {
     const float* next_scale;   // 1 value: the consumer's range, known before this layer runs
     int next_bits, next_act;
     int half_tail;             // CONV: the last k-quad of a row holds data in its first two words only
+    int tap_offset[16];        // CONV: kh * W + kw of filter tap t (pixels from the window origin); 0 past the last tap
     uint32_t pow2[24];         // pow2[e] = 2^e: branch weights read from the constant bank, so that
                                // "popcount * 2^e + acc" stays one integer multiply-add (FMA pipe)
 };
@@ -238,11 +239,9 @@ branch_kernel(const BranchParams p) {
 
     extern __shared__ uint4 smem_all[];
     __shared__ int row_n[MODE == kModeConv ? BS : 1];      // image index, or -1 for rows past the end
-    __shared__ int row_ih0[MODE == kModeConv ? BS : 1];    // top-left input coordinate of the window
-    __shared__ int row_iw0[MODE == kModeConv ? BS : 1];
     __shared__ int row_pix[MODE == kModeConv ? BS : 1];    // (n*H + ih0)*W + iw0: pixel index of the window origin
     __shared__ int row_rem[MODE == kModeConv ? BS : 1];    // oh*Wo + ow: offset of the output pixel in its plane
-    __shared__ unsigned row_out[MODE == kModeConv ? BS : 1];   // bit t set: filter tap t falls outside the image
+    __shared__ unsigned row_out[MODE == kModeConv ? BS : 1];   // bit t set: filter tap t falls outside the image (all set: no such row)
 
     chain_entry();
     const int grp = KS == 1 ? 0 : (int)threadIdx.x / 256;                 // k-group of this thread
@@ -269,14 +268,13 @@ branch_kernel(const BranchParams p) {
                 const uint32_t hw = (uint32_t)(p.Ho * p.Wo);       // output pixels fit 32 bits (checked by the host)
                 const int n = (int)((uint32_t)g / hw);
                 const int rem = (int)((uint32_t)g % hw);
+                const int ih0 = (rem / p.Wo) * p.stride - p.pad;      // top-left input coordinate of the window
+                const int iw0 = (rem % p.Wo) * p.stride - p.pad;
                 row_n[r] = n;
-                row_ih0[r] = (rem / p.Wo) * p.stride - p.pad;
-                row_iw0[r] = (rem % p.Wo) * p.stride - p.pad;
-                row_pix[r] = (n * p.H + row_ih0[r]) * p.W + row_iw0[r];
+                row_pix[r] = (n * p.H + ih0) * p.W + iw0;
                 row_rem[r] = rem;
                 // taps outside the image, bit t = tap (t / KW, t % KW).  With padding of at most one pixel only
                 // the first / last row and column of a 3 x 3 window can stick out: whole rows or columns of taps
-                const int ih0 = row_ih0[r], iw0 = row_iw0[r];
                 unsigned outside;
                 if (p.KH == 3) {
                     outside = (ih0 < 0 ? 0x007u : 0u) | (ih0 + 2 >= p.H ? 0x1C0u : 0u) |
@@ -286,8 +284,7 @@ branch_kernel(const BranchParams p) {
                 }
                 row_out[r] = outside;
             } else {
-                row_n[r] = -1; row_ih0[r] = -(1 << 20); row_iw0[r] = 0; row_pix[r] = 0;   // never inside the image
-                row_rem[r] = 0; row_out[r] = 0;
+                row_n[r] = -1; row_pix[r] = 0; row_rem[r] = 0; row_out[r] = 0xFFFFFFFFu;   // never inside the image
             }
         }
         __syncthreads();
@@ -332,16 +329,14 @@ branch_kernel(const BranchParams p) {
             constexpr int PS = (KQ * BS >= 256) ? 1 : (256 / (KQ * BS) < SB ? 256 / (KQ * BS) : SB);   // plane split
             for (int item = tid; item < KQ * BS * PS; item += 256) {
                 const int row = item % BS, kq = (item / BS) % KQ, ps = item / (BS * KQ);
-                const int ih0 = row_ih0[row], iw0 = row_iw0[row], pix0 = row_pix[row];
+                const int pix0 = row_pix[row];
+                const unsigned inside = ~row_out[row] & ((1u << (p.KH * p.KW)) - 1u);   // bit t: tap t is in the image
                 for (int part = 0; part < (1 << gs); ++part) {
                     const uint32_t copy = (uint32_t)(((kq0 + kq) << gs) + part);   // copy index along k
                     const uint32_t tap = p.tap_granules == 1 ? copy : __umulhi(copy, p.tap_magic);
                     const int cw = (int)(copy - tap * p.tap_granules) * G;
-                    const int kh = p.KW == 1 ? 0 : (int)((tap * 11u) >> 5);         // tap / 3 for tap < 9
-                    const int kw = (int)tap - kh * p.KW;
-                    const int ih = ih0 + kh, iw = iw0 + kw;
-                    const bool ok = tap < (uint32_t)(p.KH * p.KW) && ih >= 0 && ih < p.H && iw >= 0 && iw < p.W;
-                    const uint32_t* src = p.streamed + (ok ? (int64_t)(pix0 + kh * p.W + kw) * p.Cw + cw + ps * plane_words : 0);
+                    const bool ok = tap < 16u && ((inside >> tap) & 1u) != 0u;      // also false past the last tap
+                    const uint32_t* src = p.streamed + (ok ? (int64_t)(pix0 + p.tap_offset[tap & 15u]) * p.Cw + cw + ps * plane_words : 0);
                     uint32_t* dst = reinterpret_cast<uint32_t*>(ss + (ps * KQ + kq) * BS + row) + part * G;
 #pragma unroll
                     for (int plane = ps; plane < SB; plane += PS) {

@@ -164,6 +164,7 @@ extern "C" int mpq_conv_encoded(const uint32_t* x_planes, int a_bits, int N, int
     p.next_planes = next_planes; p.next_scale = next_scale; p.next_bits = next_bits; p.next_act = next_act;
     fill_pow2(p);
     p.half_tail = (ceil_div(K, 32) % 4 == 1 || ceil_div(K, 32) % 4 == 2) ? 1 : 0;
+    for (int t = 0; t < 16; ++t) p.tap_offset[t] = t < KH * KW ? (t / KW) * W + t % KW : 0;
     // held = weights (w_bits planes), streamed = activations (a_bits planes)
     return dispatch_conv(w_bits, a_bits, p, (cudaStream_t)stream);
 }
