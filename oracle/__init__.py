@@ -53,6 +53,8 @@ def _load():
             lib.mpq_oracle_gemm.restype = i64
             lib.mpq_oracle_conv.argtypes = [P, i64, i64, i64, i64, P, i64, i64, i64, i64, i64, P]
             lib.mpq_oracle_conv.restype = i64
+            lib.mpq_oracle_deconv.argtypes = [P, i64, i64, i64, i64, P, i64, i64, i64, i64, i64, P]
+            lib.mpq_oracle_deconv.restype = i64
             lib.mpq_oracle_conv_at.argtypes = [P, i64, i64, i64, P, i64, i64, i64, i64, i64, i64, i64, i64]
             lib.mpq_oracle_conv_at.restype = i64
             lib.mpq_oracle_scale.argtypes = [P, i64, i64, i64, f32, P, i32, i32, i32, P]
@@ -162,6 +164,25 @@ def conv(qx, qw, stride: int = 1, pad: int = 0) -> np.ndarray:
     return acc
 
 
+def deconv(qx, qw, stride: int = 2, pad: int = 0) -> np.ndarray:
+    """Deconvolution (transposed convolution) of decoded integers: qx [N][C][H][W], qw [O][C][KH][KW]
+    (output channel first) -> [N][O][Ho][Wo] int32 with Ho = (H - 1) stride - 2 pad + KH."""
+    qx = np.ascontiguousarray(qx, dtype=np.int16)
+    qw = np.ascontiguousarray(qw, dtype=np.int16)
+    N, C, H, W = qx.shape
+    O, C2, KH, KW = qw.shape
+    if C != C2:
+        raise ValueError("channel counts differ")
+    Ho = (H - 1) * stride - 2 * pad + KH
+    Wo = (W - 1) * stride - 2 * pad + KW
+    if Ho <= 0 or Wo <= 0:
+        raise ValueError("empty output")
+    acc = np.empty((N, O, Ho, Wo), dtype=np.int32)
+    if _load().mpq_oracle_deconv(_p(qx), N, C, H, W, _p(qw), O, KH, KW, stride, pad, _p(acc)):
+        raise OverflowError("accumulator does not fit int32")
+    return acc
+
+
 def conv_at(qx, qw, stride: int, pad: int, b: int, o: int, oh: int, ow: int) -> int:
     """One output element of :func:`conv` (for sampling a large layer)."""
     qx = np.ascontiguousarray(qx, dtype=np.int16)
@@ -237,6 +258,17 @@ def conv_layer(x, w, a_bits: int, w_bits: int, stride: int = 1, pad: int = 0,
     qx = quantize(x, s_a, a_bits, act=a_act)
     qw = quantize(w, s_w, w_bits, per_row=w_per_channel)
     acc = conv(qx, qw, stride, pad)
+    return acc, scale(acc, s_a[0], s_w, a_bits, w_bits), s_a, s_w
+
+
+def deconv_layer(x, w, a_bits: int, w_bits: int, stride: int = 2, pad: int = 0,
+                 w_per_channel: bool = True, a_act: int = HTANH):
+    """Whole encoded deconvolution layer, weights [O][C][KH][KW]: returns (acc int32, out fp32, s_a, s_w)."""
+    s_a = absmax(x, per_row=False, act=a_act)
+    s_w = absmax(w, per_row=w_per_channel)
+    qx = quantize(x, s_a, a_bits, act=a_act)
+    qw = quantize(w, s_w, w_bits, per_row=w_per_channel)
+    acc = deconv(qx, qw, stride, pad)
     return acc, scale(acc, s_a[0], s_w, a_bits, w_bits), s_a, s_w
 
 

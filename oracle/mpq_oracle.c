@@ -32,6 +32,7 @@
  */
 #include <math.h>
 #include <stdint.h>
+#include <stdlib.h>
 #include <stddef.h>
 
 /* ---- a0: scale = max |x| (NaNs ignored), per tensor or per row ----
@@ -182,6 +183,49 @@ int64_t mpq_oracle_conv(const int16_t* qx, int64_t N, int64_t C, int64_t H, int6
                     acc[((b * O + o) * Ho + oh) * Wo + ow] = (int32_t)s;
                 }
             }
+        }
+    }
+    return overflow;
+}
+
+/* ---- deconvolution (transposed convolution) on the decoded integers (Section 3.1 names the
+ * deconvolution layer among those the decomposition applies to) ----
+ * qx [N][C][H][W], qw [O][C][KH][KW] (output channel first), acc [N][O][Ho][Wo],
+ * Ho = (H - 1) stride - 2 pad + KH.  Written as the definition: every input pixel spreads its
+ * value, times the filter, over the output window that starts at (ih stride - pad, iw stride - pad);
+ * what falls outside the output is dropped.  Output positions that no input reaches stay 0. */
+int64_t mpq_oracle_deconv(const int16_t* qx, int64_t N, int64_t C, int64_t H, int64_t W,
+                          const int16_t* qw, int64_t O, int64_t KH, int64_t KW,
+                          int64_t stride, int64_t pad, int32_t* acc)
+{
+    const int64_t Ho = (H - 1) * stride - 2 * pad + KH;
+    const int64_t Wo = (W - 1) * stride - 2 * pad + KW;
+    int64_t overflow = 0;
+#pragma omp parallel for collapse(2) schedule(static) reduction(+ : overflow)
+    for (int64_t b = 0; b < N; ++b) {
+        for (int64_t o = 0; o < O; ++o) {
+            int64_t* sum = (int64_t*)calloc((size_t)(Ho * Wo), sizeof(int64_t));
+            for (int64_t c = 0; c < C; ++c) {
+                for (int64_t ih = 0; ih < H; ++ih) {
+                    for (int64_t iw = 0; iw < W; ++iw) {
+                        const int64_t v = qx[((b * C + c) * H + ih) * W + iw];
+                        for (int64_t kh = 0; kh < KH; ++kh) {
+                            const int64_t oh = ih * stride - pad + kh;
+                            if (oh < 0 || oh >= Ho) continue;
+                            for (int64_t kw = 0; kw < KW; ++kw) {
+                                const int64_t ow = iw * stride - pad + kw;
+                                if (ow < 0 || ow >= Wo) continue;
+                                sum[oh * Wo + ow] += v * (int64_t)qw[((o * C + c) * KH + kh) * KW + kw];
+                            }
+                        }
+                    }
+                }
+            }
+            for (int64_t i = 0; i < Ho * Wo; ++i) {
+                if (sum[i] > INT32_MAX || sum[i] < INT32_MIN) ++overflow;
+                acc[(b * O + o) * Ho * Wo + i] = (int32_t)sum[i];
+            }
+            free(sum);
         }
     }
     return overflow;
