@@ -190,6 +190,19 @@ def run_suite(dev: torch.device, hbm_gbs: float, path=None):
     ms = _graph_ms(lambda: mpq.encode_nchw(x, sa, 3, mpq.ACT_HRELU, out=xp))
     out["conv3x3_w3a3_32x256x14x14"]["encode_nchw_us"] = ms * 1e3
 
+    # ---- deconvolution (Section 3.1): a generator-sized upsampling layer, W4A4 ----------------------
+    N, C, H, O, ks, st, pd = 32, 256, 28, 128, 4, 2, 1
+    x, w = up(inputs.normal(34, 0, (N, C, H, H), relu=True)), up(inputs.normal(34, 1, (O, C, ks, ks), std=0.05))
+    sa, sw = mpq.absmax(x, 0, mpq.ACT_HRELU), mpq.absmax(w, mpq.SCALE_PER_ROW)
+    xp = mpq.encode_nchw(x, sa, 4, mpq.ACT_HRELU)
+    wpl, taps = mpq.encode_deconv_weights(w, sw, 4, st)
+    Ho = (H - 1) * st - 2 * pd + ks
+    yf = torch.empty((N, O, Ho, Ho), dtype=torch.float32, device=dev)
+    ms = _graph_ms(lambda: mpq.deconv(xp, 4, N, C, H, H, wpl, 4, taps, O, ks, ks, st, pd, None, yf, sa, sw, mpq.SCALE_PER_ROW))
+    M, K = N * Ho * Ho, (ks // st) * (ks // st) * C                # every output sums 2 x 2 taps x C products
+    out["deconv4x4s2_w4a4_32x256x28x28"] = product_record(ms, M, O, K, 4, 4, 16.0 * M * O * (K // 32))
+    del x, w, yf
+
     # ---- workload 5: ResNet-18-shaped stack, W4A4, batch 128 -------------------------------------
     batch = 128
     net = QuantResNet18Stack(inputs.config5_weights(), batch, 224, 4, 4, dev)
@@ -259,7 +272,7 @@ def compact(d: dict) -> dict:
     c = {"peaks": {"mix_peak_gpopc_s": r3(d["branch_peak_gpopc_s"]), "plain_popc_gpopc_s": r3(d["popc_peak_gpopc_s"]),
                    "hbm_gbs": d["hbm_gbs"]},
          "gemm_w2a2_64x64x512": {"us": r3(d["gemm_w2a2_64x64x512"]["us"])}}
-    for name in ("fc_w2a2_64x4096x9216", "conv3x3_w3a3_32x256x14x14"):
+    for name in ("fc_w2a2_64x4096x9216", "conv3x3_w3a3_32x256x14x14", "deconv4x4s2_w4a4_32x256x28x28"):
         r = d[name]
         c[name] = {"us": r3(r["ms"] * 1e3), "equivalent_tops": r3(r["equivalent_tops"]), "frac": r3(r["frac_of_branch_peak"])}
     c["conv3x3_w3a3_32x256x14x14"]["encode_nchw_us"] = r3(d["conv3x3_w3a3_32x256x14x14"]["encode_nchw_us"])
@@ -314,6 +327,9 @@ def summary_markdown(d: dict) -> str:
     r = d["conv3x3_w3a3_32x256x14x14"]
     L.append("| conv 3x3 W3A3 32x256x14x14 -> 256 (fp32 out) | %.1f us (+ encode_nchw %.1f us) | %.1f | %.3f | %.3f |"
              % (r["ms"] * 1e3, r["encode_nchw_us"], r["equivalent_tops"], r["frac_of_branch_peak"], r["frac_of_plain_popc_peak"]))
+    r = d["deconv4x4s2_w4a4_32x256x28x28"]
+    L.append("| deconv 4x4 stride 2 W4A4 32x256x28x28 -> 128 x 56 x 56 (fp32 out, one launch per output phase) | %.1f us | %.1f | %.3f | %.3f |"
+             % (r["ms"] * 1e3, r["equivalent_tops"], r["frac_of_branch_peak"], r["frac_of_plain_popc_peak"]))
     s = d["resnet18_stack_w4a4_b128"]
     L += ["\n## ResNet-18-shaped stack, W4A4, batch 128, 224 x 224\n",
           "%.2f ms per step = **%.0f images/s** end to end (fp32 stem + max-pool + 19 encoded convolutions; residual add,"
@@ -347,6 +363,7 @@ def _single(argv):
         python bench_suite.py gemm A_BITS W_BITS SIZE
         python bench_suite.py conv BITS N C HW O KSIZE STRIDE
         python bench_suite.py fc A_BITS W_BITS M N K
+        python bench_suite.py deconv BITS N C HW O KSIZE STRIDE PAD
         python bench_suite.py encode BITS ROWS K            (row encoder, four inputs in rotation)
         python bench_suite.py nchw BITS N C HW              (NCHW encoder)
         python bench_suite.py absmax ROWS K
@@ -376,6 +393,18 @@ def _single(argv):
         fn = lambda: mpq.conv(xp, bits, N, C, HW, HW, wp, bits, taps, O, ks, ks, stride, pad, None, y, sa, sw,
                               mpq.SCALE_PER_ROW)
         popcs = float(bits * bits) * N * Ho * Ho * O * (ks * ks * C // 32)
+    elif argv[0] == "deconv":
+        bits, N, C, HW, O, ks, stride, pad = (int(a) for a in argv[1:9])
+        x = torch.randn(N, C, HW, HW, device=dev).relu_()
+        w = torch.randn(O, C, ks, ks, device=dev)
+        sa, sw = mpq.absmax(x, 0, mpq.ACT_HRELU), mpq.absmax(w, mpq.SCALE_PER_ROW)
+        xp = mpq.encode_nchw(x, sa, bits, mpq.ACT_HRELU)
+        wp, taps = mpq.encode_deconv_weights(w, sw, bits, stride)
+        Ho = (HW - 1) * stride - 2 * pad + ks
+        y = torch.empty((N, O, Ho, Ho), dtype=torch.float32, device=dev)
+        fn = lambda: mpq.deconv(xp, bits, N, C, HW, HW, wp, bits, taps, O, ks, ks, stride, pad, None, y, sa, sw,
+                                mpq.SCALE_PER_ROW)
+        popcs = float(bits * bits) * N * HW * HW * O * (ks * ks * C // 32)   # every input pixel meets every tap once
     elif argv[0] == "fc":
         ab, wb, m, n, k = (int(a) for a in argv[1:6])
         x = torch.randn(m, k, device=dev).relu_()

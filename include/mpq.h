@@ -176,6 +176,36 @@ int mpq_conv_fused(const uint32_t* x_planes, int a_bits, int N, int C, int H, in
                    const float* x_scale, const float* w_scale, int w_mode,
                    const float* residual, int relu, float* out_max, void* stream);
 
+/* ---- Deconvolution (transposed convolution) by the same decomposition (Section 3.1 names the
+ * deconvolution layer, next to the fully connected and the convolution layer, as one the method
+ * applies to).  y[n][o][oh][ow] = sum over (c, kh, kw, ih, iw) with oh = ih*stride - pad + kh and
+ * ow = iw*stride - pad + kw of q_x[n][c][ih][iw] * q_w[o][c][kh][kw]; y is [N][O][Ho][Wo] with
+ * Ho = (H-1)*stride - 2*pad + KH.  Outputs that share (oh mod stride, ow mod stride) use the same
+ * taps, so the layer runs as stride^2 gathers on the packed planes, one per output phase, each with
+ * the branch kernel of mpq_conv; an output position that no input reaches gets 0.
+ * Filters: stride 1 or 2, stride <= KH, KW <= 4, 0 <= pad < min(KH, KW); C as for mpq_conv.
+ *
+ * Weights: w [O][C][KH][KW] fp32 (OUTPUT channel first; a framework that stores transposed-
+ * convolution filters input channel first swaps the two axes when it hands them over).
+ * mpq_encode_deconv_weights writes mpq_deconv_weight_words() words: for each filter phase
+ * (r_h, r_w) = (kh mod stride, kw mod stride), in the order r_h*stride + r_w, a matrix
+ * [bits][O][mpq_row_words(T_h*T_w*C)] whose row o holds the taps kh = r_h + stride*t_h,
+ * kw = r_w + stride*t_w ordered (t_h, t_w, c); and tap_sums [KH*KW][O] int32 (sum over c of the
+ * decoded weight, taps counted phase by phase in that same order).  scale: 1 value or O values.
+ * mpq_deconv_weight_words returns 0 for arguments outside the limits above. */
+int64_t mpq_deconv_weight_words(int O, int C, int KH, int KW, int stride, int bits);
+int mpq_encode_deconv_weights(const float* w, int O, int C, int KH, int KW, int stride,
+                              const float* scale, int mode, int bits,
+                              uint32_t* planes, int32_t* tap_sums, void* stream);
+/* x_planes from mpq_encode_nchw.  y_i32 / y_f32: either may be NULL, not both.  residual, relu and
+ * out_max as in mpq_conv_fused (they need y_f32). */
+int mpq_deconv(const uint32_t* x_planes, int a_bits, int N, int C, int H, int W,
+               const uint32_t* w_planes, int w_bits, const int32_t* tap_sums,
+               int O, int KH, int KW, int stride, int pad,
+               int32_t* y_i32, float* y_f32,
+               const float* x_scale, const float* w_scale, int w_mode,
+               const float* residual, int relu, float* out_max, void* stream);
+
 /* mpq_conv_fused that also runs the CONSUMER's Encoder in its store (Fig. 1: the Decoder of one
  * layer feeding the Encoder of the next), for networks whose ranges are known before the layer
  * runs: the paper's fixed HReLU range [0,1] (Table 1), or a calibrated constant.  The value f

@@ -62,6 +62,11 @@ def lib() -> ctypes.CDLL:
         L.mpq_maxpool3x3s2.argtypes = [P, P, i32, i32, i32, i32, P, P]
         L.mpq_conv_fused.argtypes = [P, i32, i32, i32, i32, i32, P, i32, P, i32, i32, i32, i32, i32, P, P, P, P, i32,
                                      P, i32, P, P]
+        L.mpq_deconv.argtypes = [P, i32, i32, i32, i32, i32, P, i32, P, i32, i32, i32, i32, i32, P, P, P, P, i32,
+                                 P, i32, P, P]
+        L.mpq_deconv_weight_words.argtypes = [i32, i32, i32, i32, i32, i32]
+        L.mpq_deconv_weight_words.restype = i64
+        L.mpq_encode_deconv_weights.argtypes = [P, i32, i32, i32, i32, i32, P, i32, i32, P, P, P]
         L.mpq_zero.argtypes = [P, i64, P]
         L.mpq_linear_workspace.argtypes = [i64, i64, i64, i32, i32]
         L.mpq_linear_workspace.restype = i64
@@ -83,7 +88,8 @@ def lib() -> ctypes.CDLL:
         L.mpq_measure_b1_mma_peak.restype = i32
         for name in ("mpq_absmax", "mpq_encode", "mpq_encode_nchw", "mpq_encode_oihw", "mpq_gemm", "mpq_conv",
                      "mpq_add_relu", "mpq_stem_conv7x7", "mpq_maxpool3x3s2", "mpq_conv_fused", "mpq_zero", "mpq_linear", "mpq_linear_static", "mpq_linear_host", "mpq_measure_popc_peak",
-                     "mpq_encode_with", "mpq_encode_ranged", "mpq_gemm_fused", "mpq_conv_encoded", "mpq_linear_host_prepared"):
+                     "mpq_encode_with", "mpq_encode_ranged", "mpq_gemm_fused", "mpq_conv_encoded", "mpq_linear_host_prepared",
+                     "mpq_deconv", "mpq_encode_deconv_weights"):
             getattr(L, name).restype = i32
         _lib = L
     return _lib
@@ -268,6 +274,38 @@ def conv_encoded(x_planes: torch.Tensor, a_bits: int, N: int, C: int, H: int, W:
                                   _ptr(next_scale, torch.float32), next_act, next_bits,
                                   _ptr(next_planes, torch.int32), _stream()), "mpq_conv_encoded")
     return next_planes
+
+
+def encode_deconv_weights(w: torch.Tensor, scale: torch.Tensor, bits: int, stride: int, mode: int = SCALE_PER_ROW):
+    """Deconvolution filters [O][C][KH][KW] fp32 (output channel first) -> (planes, one packed matrix per
+    filter phase, flat int32; tap_sums [KH*KW][O], taps counted phase by phase)."""
+    O, C, KH, KW = w.shape
+    words = lib().mpq_deconv_weight_words(O, C, KH, KW, stride, bits)
+    if words <= 0:
+        raise MpqError(3, "mpq_deconv_weight_words")          # MPQ_ERR_UNSUPPORTED: filter outside the supported set
+    planes = torch.empty((words,), dtype=torch.int32, device=w.device)
+    tap_sums = torch.empty((KH * KW, O), dtype=torch.int32, device=w.device)
+    _check(lib().mpq_encode_deconv_weights(_ptr(w, torch.float32), O, C, KH, KW, stride, _ptr(scale, torch.float32),
+                                           mode, bits, _ptr(planes, torch.int32), _ptr(tap_sums, torch.int32),
+                                           _stream()), "mpq_encode_deconv_weights")
+    return planes, tap_sums
+
+
+def deconv(x_planes: torch.Tensor, a_bits: int, N: int, C: int, H: int, W: int,
+           w_planes: torch.Tensor, w_bits: int, tap_sums: torch.Tensor,
+           O: int, KH: int, KW: int, stride: int, pad: int,
+           y_i32: Optional[torch.Tensor], y_f32: Optional[torch.Tensor],
+           x_scale: Optional[torch.Tensor] = None, w_scale: Optional[torch.Tensor] = None,
+           w_mode: int = SCALE_PER_ROW, residual: Optional[torch.Tensor] = None, relu: bool = False,
+           out_max: Optional[torch.Tensor] = None):
+    """Deconvolution (transposed convolution) on packed planes -> [N][O][Ho][Wo], Ho = (H-1)*stride - 2*pad + KH."""
+    _check(lib().mpq_deconv(_ptr(x_planes, torch.int32), a_bits, N, C, H, W, _ptr(w_planes, torch.int32), w_bits,
+                            _ptr(tap_sums, torch.int32), O, KH, KW, stride, pad,
+                            _ptr(y_i32, torch.int32), _ptr(y_f32, torch.float32),
+                            _ptr(x_scale, torch.float32), _ptr(w_scale, torch.float32), w_mode,
+                            _ptr(residual, torch.float32), int(relu), _ptr(out_max, torch.float32), _stream()),
+           "mpq_deconv")
+    return y_i32, y_f32
 
 
 def zero(t: torch.Tensor) -> torch.Tensor:

@@ -58,7 +58,15 @@ struct BranchParams {
     const float* next_scale;   // 1 value: the consumer's range, known before this layer runs
     int next_bits, next_act;
     int half_tail;             // CONV: the last k-quad of a row holds data in its first two words only
-    int tap_offset[16];        // CONV: kh * W + kw of filter tap t (pixels from the window origin); 0 past the last tap
+    int tap_offset[16];        // CONV: dh * W + dw of filter tap t (pixels from the window origin); 0 past the last tap
+    // CONV: the pixels of this launch form a sub_h x sub_w grid per image.  Grid point (a, b) has its window
+    // origin at input pixel (a * in_step + in_h0, b * in_step + in_w0), tap t reads the pixel (tap_dh[t],
+    // tap_dw[t]) away from it, and the result goes to output pixel (out_h0 + a * out_step, out_w0 + b * out_step)
+    // of the Ho x Wo output.  A convolution: in_step = stride, in_h0 = -pad, taps (kh, kw), the whole output.
+    // A deconvolution runs one launch per output phase: in_step = 1, taps (-th, -tw), out_step = stride.
+    int sub_h, sub_w, in_step, in_h0, in_w0, out_h0, out_w0, out_step;
+    int window3x3;             // taps are (kh, kw) of a 3 x 3 window that sticks out by at most one pixel
+    signed char tap_dh[16], tap_dw[16];
     uint32_t pow2[24];         // pow2[e] = 2^e: branch weights read from the constant bank, so that
                                // "popcount * 2^e + acc" stays one integer multiply-add (FMA pipe)
 };
@@ -265,22 +273,26 @@ branch_kernel(const BranchParams p) {
         for (int r = tid; r < BS; r += 256) {
             const int64_t g = s0 + r;
             if (g < p.streamed_rows) {
-                const uint32_t hw = (uint32_t)(p.Ho * p.Wo);       // output pixels fit 32 bits (checked by the host)
-                const int n = (int)((uint32_t)g / hw);
-                const int rem = (int)((uint32_t)g % hw);
-                const int ih0 = (rem / p.Wo) * p.stride - p.pad;      // top-left input coordinate of the window
-                const int iw0 = (rem % p.Wo) * p.stride - p.pad;
+                const uint32_t shw = (uint32_t)(p.sub_h * p.sub_w);  // pixels fit 32 bits (checked by the host)
+                const int n = (int)((uint32_t)g / shw);
+                const int srem = (int)((uint32_t)g % shw);
+                const int ga = srem / p.sub_w, gb = srem % p.sub_w;
+                const int ih0 = ga * p.in_step + p.in_h0;             // input coordinate of the window origin
+                const int iw0 = gb * p.in_step + p.in_w0;
                 row_n[r] = n;
                 row_pix[r] = (n * p.H + ih0) * p.W + iw0;
-                row_rem[r] = rem;
-                // taps outside the image, bit t = tap (t / KW, t % KW).  With padding of at most one pixel only
-                // the first / last row and column of a 3 x 3 window can stick out: whole rows or columns of taps
-                unsigned outside;
-                if (p.KH == 3) {
+                row_rem[r] = (p.out_h0 + ga * p.out_step) * p.Wo + p.out_w0 + gb * p.out_step;
+                // taps outside the image, bit t = tap t.  A 3 x 3 window with padding of at most one pixel: only
+                // its first / last row and column can stick out, whole rows or columns of taps at once
+                unsigned outside = 0u;
+                if (p.window3x3) {
                     outside = (ih0 < 0 ? 0x007u : 0u) | (ih0 + 2 >= p.H ? 0x1C0u : 0u) |
                               (iw0 < 0 ? 0x049u : 0u) | (iw0 + 2 >= p.W ? 0x124u : 0u);
                 } else {
-                    outside = (ih0 < 0 || ih0 >= p.H || iw0 < 0 || iw0 >= p.W) ? 1u : 0u;
+                    for (int t = 0; t < p.KH * p.KW; ++t) {
+                        const int ih = ih0 + p.tap_dh[t], iw = iw0 + p.tap_dw[t];
+                        if (ih < 0 || ih >= p.H || iw < 0 || iw >= p.W) outside |= 1u << t;
+                    }
                 }
                 row_out[r] = outside;
             } else {

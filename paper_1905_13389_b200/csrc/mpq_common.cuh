@@ -14,6 +14,33 @@ __host__ __device__ inline int64_t ceil_div(int64_t a, int64_t b) { return (a + 
 // Words per packed row: ceil(k/32) rounded up to 4 words (16 bytes).
 __host__ __device__ inline int64_t row_words(int64_t k) { return ceil_div(ceil_div(k, 32), 4) * 4; }
 
+// Deconvolution weights are stored as one packed matrix per filter phase (r_h, r_w) = (kh mod stride,
+// kw mod stride): the taps kh = r_h + stride * t_h, kw = r_w + stride * t_w that reach the same output
+// phase, k ordered (t_h, t_w, c).  Phases in the order r_h * stride + r_w, each [bits][O][rw].
+inline bool deconv_filter_ok(int KH, int KW, int stride) {
+    return (stride == 1 || stride == 2) && KH >= stride && KW >= stride && KH <= 4 && KW <= 4;
+}
+struct DeconvPhase {
+    int r_h, r_w, T_h, T_w;      // phase and its tap counts
+    int tap_start;               // first row of its tap sums (taps counted phase by phase)
+    int64_t rw;                  // words per packed row = row_words(T_h * T_w * C)
+    int64_t word_offset;         // where its planes start
+};
+inline int64_t deconv_phases(int O, int C, int KH, int KW, int stride, int bits, DeconvPhase (&ph)[4]) {
+    int64_t words = 0;
+    int taps = 0, n = 0;
+    for (int r_h = 0; r_h < stride; ++r_h)
+        for (int r_w = 0; r_w < stride; ++r_w) {
+            DeconvPhase& g = ph[n++];
+            g.r_h = r_h; g.r_w = r_w;
+            g.T_h = (KH - r_h + stride - 1) / stride; g.T_w = (KW - r_w + stride - 1) / stride;
+            g.tap_start = taps; taps += g.T_h * g.T_w;
+            g.rw = row_words((int64_t)g.T_h * g.T_w * C);
+            g.word_offset = words; words += (int64_t)bits * O * g.rw;
+        }
+    return words;
+}
+
 inline bool bits_ok(int b) { return b >= 1 && b <= kMaxBits; }
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 

@@ -428,7 +428,20 @@ __device__ __forceinline__ int level_index_rt(float x, float inv, int bits) {
     return level_index<ACT>(x, inv, 0.5f * (float)((1 << bits) - 1), (float)(-H), (float)H - 0.5f, H);
 }
 
-__global__ void encode_oihw_kernel(const float* __restrict__ w, int O, int C, int taps,
+// The row of output channel o holds `taps` filter taps; tap t of the row is tap map.from[t] of the
+// filter's KH*KW (the identity for a convolution, one phase's taps for a deconvolution).
+struct TapMap {
+    int filter_taps;          // KH * KW
+    int from[16];
+};
+static TapMap identity_taps(int taps) {
+    TapMap m;
+    m.filter_taps = taps;
+    for (int t = 0; t < 16; ++t) m.from[t] = t < taps ? t : 0;
+    return m;
+}
+
+__global__ void encode_oihw_kernel(const float* __restrict__ w, int O, int C, int taps, const TapMap map,
                                    const float* __restrict__ scale, int per_row, int bits,
                                    uint32_t* __restrict__ planes, int64_t rw) {
     const int64_t id = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -443,13 +456,13 @@ __global__ void encode_oihw_kernel(const float* __restrict__ w, int O, int C, in
         const int64_t kidx = word * 32 + t;
         if (kidx >= K) break;
         const int64_t tap = kidx / C, c = kidx % C;
-        const uint32_t u = (uint32_t)level_index_rt<MPQ_ACT_HTANH>(__ldg(w + (o * C + c) * taps + tap), inv, bits);
+        const uint32_t u = (uint32_t)level_index_rt<MPQ_ACT_HTANH>(__ldg(w + (o * C + c) * map.filter_taps + map.from[tap]), inv, bits);
         for (int p = 0; p < kMaxBits; ++p) out[p] |= ((u >> p) & 1u) << t;
     }
     for (int p = 0; p < bits; ++p) planes[((int64_t)p * O + o) * rw + word] = out[p];
 }
 
-__global__ void tap_sums_kernel(const float* __restrict__ w, int O, int C, int taps,
+__global__ void tap_sums_kernel(const float* __restrict__ w, int O, int C, int taps, const TapMap map,
                                 const float* __restrict__ scale, int per_row, int bits,
                                 int32_t* __restrict__ tap_sums) {
     const int64_t id = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -459,7 +472,7 @@ __global__ void tap_sums_kernel(const float* __restrict__ w, int O, int C, int t
     const int L = (1 << bits) - 1;
     int32_t s = 0;
     for (int c = 0; c < C; ++c)
-        s += 2 * level_index_rt<MPQ_ACT_HTANH>(__ldg(w + (o * C + c) * taps + tap), inv, bits) - L;
+        s += 2 * level_index_rt<MPQ_ACT_HTANH>(__ldg(w + (o * C + c) * map.filter_taps + map.from[tap]), inv, bits) - L;
     tap_sums[tap * O + o] = s;
 }
 
@@ -597,20 +610,55 @@ extern "C" int mpq_encode_nchw(const float* x, int N, int C, int H, int W, const
     return dispatch_bits_act<EncodeNchwLauncher>(bits, act, x, N, C, (int64_t)H * W, scale, planes, (cudaStream_t)stream);
 }
 
+static int encode_filter_rows(const float* w, int O, int C, int taps, const TapMap& map, const float* scale,
+                              int per_row, int bits, uint32_t* planes, int32_t* tap_sums, cudaStream_t st) {
+    const int64_t rw = row_words((int64_t)taps * C);
+    encode_oihw_kernel<<<(unsigned)ceil_div((int64_t)O * rw, 128), 128, 0, st>>>(w, O, C, taps, map, scale, per_row, bits, planes, rw);
+    if (launch_status() != MPQ_OK) return MPQ_ERR_CUDA;
+    tap_sums_kernel<<<(unsigned)ceil_div((int64_t)O * taps, 128), 128, 0, st>>>(w, O, C, taps, map, scale, per_row, bits, tap_sums);
+    return launch_status();
+}
+
 extern "C" int mpq_encode_oihw(const float* w, int O, int C, int KH, int KW, const float* scale, int mode,
                                int bits, uint32_t* planes, int32_t* tap_sums, void* stream) {
     if (!w || !scale || !planes || !tap_sums) return MPQ_ERR_NULL;
     if (O <= 0 || C <= 0 || KH <= 0 || KW <= 0) return MPQ_ERR_BAD_SHAPE;
     if (!bits_ok(bits) || !conv_channels_ok(C) || (mode != MPQ_SCALE_PER_TENSOR && mode != MPQ_SCALE_PER_ROW)) return MPQ_ERR_UNSUPPORTED;
     if (!aligned16(planes)) return MPQ_ERR_ALIGN;
-    cudaStream_t st = (cudaStream_t)stream;
-    const int taps = KH * KW;
-    const int64_t rw = row_words((int64_t)taps * C);
-    const int per_row = mode == MPQ_SCALE_PER_ROW;
-    encode_oihw_kernel<<<(unsigned)ceil_div((int64_t)O * rw, 128), 128, 0, st>>>(w, O, C, taps, scale, per_row, bits, planes, rw);
-    if (launch_status() != MPQ_OK) return MPQ_ERR_CUDA;
-    tap_sums_kernel<<<(unsigned)ceil_div((int64_t)O * taps, 128), 128, 0, st>>>(w, O, C, taps, scale, per_row, bits, tap_sums);
-    return launch_status();
+    if (KH * KW > 16) return MPQ_ERR_UNSUPPORTED;
+    return encode_filter_rows(w, O, C, KH * KW, identity_taps(KH * KW), scale, mode == MPQ_SCALE_PER_ROW, bits,
+                              planes, tap_sums, (cudaStream_t)stream);
+}
+
+extern "C" int64_t mpq_deconv_weight_words(int O, int C, int KH, int KW, int stride, int bits) {
+    if (O <= 0 || C <= 0 || KH <= 0 || KW <= 0 || !bits_ok(bits) || !deconv_filter_ok(KH, KW, stride)) return 0;
+    DeconvPhase ph[4];
+    return deconv_phases(O, C, KH, KW, stride, bits, ph);
+}
+
+extern "C" int mpq_encode_deconv_weights(const float* w, int O, int C, int KH, int KW, int stride,
+                                         const float* scale, int mode, int bits,
+                                         uint32_t* planes, int32_t* tap_sums, void* stream) {
+    if (!w || !scale || !planes || !tap_sums) return MPQ_ERR_NULL;
+    if (O <= 0 || C <= 0 || KH <= 0 || KW <= 0) return MPQ_ERR_BAD_SHAPE;
+    if (!bits_ok(bits) || !conv_channels_ok(C) || !deconv_filter_ok(KH, KW, stride) ||
+        (mode != MPQ_SCALE_PER_TENSOR && mode != MPQ_SCALE_PER_ROW)) return MPQ_ERR_UNSUPPORTED;
+    if (!aligned16(planes)) return MPQ_ERR_ALIGN;
+    DeconvPhase ph[4];
+    deconv_phases(O, C, KH, KW, stride, bits, ph);
+    for (int g = 0; g < stride * stride; ++g) {
+        TapMap map;
+        map.filter_taps = KH * KW;
+        for (int t = 0; t < 16; ++t) map.from[t] = 0;
+        for (int t_h = 0; t_h < ph[g].T_h; ++t_h)
+            for (int t_w = 0; t_w < ph[g].T_w; ++t_w)
+                map.from[t_h * ph[g].T_w + t_w] = (ph[g].r_h + stride * t_h) * KW + ph[g].r_w + stride * t_w;
+        const int rc = encode_filter_rows(w, O, C, ph[g].T_h * ph[g].T_w, map, scale, mode == MPQ_SCALE_PER_ROW, bits,
+                                          planes + ph[g].word_offset, tap_sums + (int64_t)ph[g].tap_start * O,
+                                          (cudaStream_t)stream);
+        if (rc != MPQ_OK) return rc;
+    }
+    return MPQ_OK;
 }
 
 extern "C" int mpq_add_relu(const float* a, const float* b, float* y, int64_t n, void* stream) {

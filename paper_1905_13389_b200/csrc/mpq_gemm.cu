@@ -164,7 +164,82 @@ extern "C" int mpq_conv_encoded(const uint32_t* x_planes, int a_bits, int N, int
     p.next_planes = next_planes; p.next_scale = next_scale; p.next_bits = next_bits; p.next_act = next_act;
     fill_pow2(p);
     p.half_tail = (ceil_div(K, 32) % 4 == 1 || ceil_div(K, 32) % 4 == 2) ? 1 : 0;
-    for (int t = 0; t < 16; ++t) p.tap_offset[t] = t < KH * KW ? (t / KW) * W + t % KW : 0;
+    for (int t = 0; t < 16; ++t) {
+        const bool live = t < KH * KW;
+        p.tap_dh[t] = (signed char)(live ? t / KW : 0);
+        p.tap_dw[t] = (signed char)(live ? t % KW : 0);
+        p.tap_offset[t] = p.tap_dh[t] * W + p.tap_dw[t];
+    }
+    p.sub_h = p.Ho; p.sub_w = p.Wo; p.in_step = stride; p.in_h0 = -pad; p.in_w0 = -pad;
+    p.out_h0 = 0; p.out_w0 = 0; p.out_step = 1;
+    p.window3x3 = KH == 3 ? 1 : 0;
     // held = weights (w_bits planes), streamed = activations (a_bits planes)
     return dispatch_conv(w_bits, a_bits, p, (cudaStream_t)stream);
+}
+
+// Deconvolution: output pixel (oh, ow) receives x[ih][iw] * w[kh][kw] from every (ih, kh) with
+// oh = ih * stride - pad + kh.  Outputs of one phase (oh mod stride, ow mod stride) all use the same
+// taps, kh = r_h + stride * t_h with r_h = (oh + pad) mod stride, and ih = (oh + pad - r_h) / stride - t_h:
+// per phase an ordinary gather over a T_h x T_w window that steps backwards through the image.  One
+// launch of the branch kernel per phase, each over that phase's part of the output.
+extern "C" int mpq_deconv(const uint32_t* x_planes, int a_bits, int N, int C, int H, int W,
+                          const uint32_t* w_planes, int w_bits, const int32_t* tap_sums,
+                          int O, int KH, int KW, int stride, int pad,
+                          int32_t* y_i32, float* y_f32,
+                          const float* x_scale, const float* w_scale, int w_mode,
+                          const float* residual, int relu, float* out_max, void* stream) {
+    if ((residual || relu || out_max) && !y_f32) return MPQ_ERR_NULL;
+    if (!x_planes || !w_planes || !tap_sums || (!y_i32 && !y_f32)) return MPQ_ERR_NULL;
+    if (y_f32 && (!x_scale || !w_scale)) return MPQ_ERR_NULL;
+    if (N <= 0 || C <= 0 || H <= 0 || W <= 0 || O <= 0 || KH <= 0 || KW <= 0) return MPQ_ERR_BAD_SHAPE;
+    if (!bits_ok(a_bits) || !bits_ok(w_bits) || !deconv_filter_ok(KH, KW, stride) || pad < 0 || pad >= KH || pad >= KW ||
+        !(C == 32 || C == 64 || C % 128 == 0) ||
+        (w_mode != MPQ_SCALE_PER_TENSOR && w_mode != MPQ_SCALE_PER_ROW)) return MPQ_ERR_UNSUPPORTED;
+    const int Ho = (H - 1) * stride - 2 * pad + KH, Wo = (W - 1) * stride - 2 * pad + KW;
+    if (Ho <= 0 || Wo <= 0) return MPQ_ERR_BAD_SHAPE;
+    if (!aligned16(x_planes) || !aligned16(w_planes)) return MPQ_ERR_ALIGN;
+    // an output sums at most ceil(KH/stride) * ceil(KW/stride) * C products
+    const int64_t k_max = (int64_t)ceil_div(KH, stride) * ceil_div(KW, stride) * C;
+    if (!int32_headroom(k_max, a_bits, w_bits)) return MPQ_ERR_OVERFLOW;
+    if ((int64_t)N * H * W >= ((int64_t)1 << 31) || (int64_t)N * Ho * Wo >= ((int64_t)1 << 31)) return MPQ_ERR_UNSUPPORTED;
+    DeconvPhase phases[4];
+    deconv_phases(O, C, KH, KW, stride, w_bits, phases);
+    for (int out_ph = 0; out_ph < stride; ++out_ph) {
+        for (int out_pw = 0; out_pw < stride; ++out_pw) {
+            if (out_ph >= Ho || out_pw >= Wo) continue;                     // no output in this phase
+            const int r_h = (out_ph + pad) % stride, r_w = (out_pw + pad) % stride;
+            const DeconvPhase& g = phases[r_h * stride + r_w];
+            BranchParams p = {};
+            p.held = w_planes + g.word_offset; p.streamed = x_planes;
+            p.Ho = Ho; p.Wo = Wo;
+            p.sub_h = (int)ceil_div(Ho - out_ph, stride); p.sub_w = (int)ceil_div(Wo - out_pw, stride);
+            p.held_rows = O; p.held_plane_rows = O; p.streamed_rows = (int64_t)N * p.sub_h * p.sub_w;
+            p.k = (int64_t)g.T_h * g.T_w * C; p.rw = g.rw;
+            p.out_i32 = y_i32; p.out_f32 = y_f32; p.ldc = 0;
+            p.a_scale = x_scale; p.w_scale = w_scale; p.w_per_row = w_mode == MPQ_SCALE_PER_ROW;
+            p.N = N; p.C = C; p.H = H; p.W = W; p.O = O; p.KH = g.T_h; p.KW = g.T_w; p.stride = stride; p.pad = pad;
+            p.Cw = C / 32; p.granule = p.Cw >= 4 ? 4 : p.Cw;
+            p.granule_shift = p.granule == 4 ? 0 : p.granule == 2 ? 1 : 2;
+            p.tap_granules = p.Cw / p.granule;
+            p.tap_magic = p.tap_granules > 1 ? (uint32_t)((((uint64_t)1 << 32) + p.tap_granules - 1) / p.tap_granules) : 0u;
+            if ((p.rw << p.granule_shift) >= 65536) return MPQ_ERR_UNSUPPORTED;
+            p.tap_sums = tap_sums + (int64_t)g.tap_start * O;
+            p.residual = residual; p.relu = relu != 0; p.out_max = out_max;
+            fill_pow2(p);
+            const int64_t kw32 = ceil_div(p.k, 32);
+            p.half_tail = (kw32 % 4 == 1 || kw32 % 4 == 2) ? 1 : 0;
+            for (int t = 0; t < 16; ++t) {
+                const bool live = t < g.T_h * g.T_w;
+                p.tap_dh[t] = (signed char)(live ? -(t / g.T_w) : 0);
+                p.tap_dw[t] = (signed char)(live ? -(t % g.T_w) : 0);
+                p.tap_offset[t] = p.tap_dh[t] * W + p.tap_dw[t];
+            }
+            p.in_step = 1; p.in_h0 = (out_ph + pad - r_h) / stride; p.in_w0 = (out_pw + pad - r_w) / stride;
+            p.out_h0 = out_ph; p.out_w0 = out_pw; p.out_step = stride;
+            p.window3x3 = 0;
+            const int rc = dispatch_conv(w_bits, a_bits, p, (cudaStream_t)stream);
+            if (rc != MPQ_OK) return rc;
+        }
+    }
+    return MPQ_OK;
 }
