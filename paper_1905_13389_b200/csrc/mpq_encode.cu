@@ -15,6 +15,11 @@ constexpr int kAbsmaxThreads = 256;
 constexpr int kAbsmaxChunk = 8192;  // elements per CTA and step
 constexpr int kAbsmaxPerSm = 6;     // CTAs per multiprocessor: 6 x 32 KiB of loads in flight
 
+__global__ void zero_floats_kernel(float* __restrict__ p, int64_t n) {
+    chain_entry();
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) p[i] = 0.0f;
+}
+
 // The grid is at most a few CTAs per multiprocessor; every CTA walks the chunks of the tensor in
 // a grid-stride loop, so all multiprocessors finish together whatever the tensor's size.
 template <int ACT, bool VEC4>
@@ -559,7 +564,13 @@ extern "C" int mpq_absmax(const float* x, int64_t rows, int64_t k, int64_t ldx, 
         (act != MPQ_ACT_HTANH && act != MPQ_ACT_HRELU)) return MPQ_ERR_UNSUPPORTED;
     cudaStream_t st = (cudaStream_t)stream;
     const int per_row = mode == MPQ_SCALE_PER_ROW;
-    if (cudaMemsetAsync(scale_out, 0, sizeof(float) * (per_row ? rows : 1), st) != cudaSuccess) return MPQ_ERR_CUDA;
+    // zeroed by a kernel of the chain rather than a memset node: the range kernel's blocks are then
+    // already resident (waiting at their chain entry) when the zeroes land
+    {
+        const int64_t n = per_row ? rows : 1;
+        const int rc = launch_chained_as(true, zero_floats_kernel, (unsigned)min(ceil_div(n, 256), (int64_t)1024), 256, 0, st, scale_out, n);
+        if (rc != MPQ_OK) return rc;
+    }
     if (!per_row && ldx == k) { k = rows * k; ldx = k; rows = 1; }   // contiguous tensor: one long row
     const int64_t chunks = ceil_div(k, kAbsmaxChunk);
     const int64_t total = rows * chunks;
