@@ -122,7 +122,7 @@ int mpq_encode_nchw(const float* x, int N, int C, int H, int W, const float* sca
 /* Weights for mpq_conv: w [O][C][KH][KW] fp32 -> planes[bits][O][mpq_row_words(KH*KW*C)], the
  * row of output channel o ordered (kh, kw, c) with c innermost.  scale: 1 value or O values.
  * tap_sums [KH*KW][O] int32 (required): sum over c of the decoded weight q_w[o][c][kh][kw];
- * mpq_conv uses it to make out-of-image taps contribute exactly 0. */
+ * mpq_conv uses it to make out-of-image taps contribute exactly 0.  KH*KW <= 16. */
 int mpq_encode_oihw(const float* w, int O, int C, int KH, int KW, const float* scale, int mode,
                     int bits, uint32_t* planes, int32_t* tap_sums, void* stream);
 

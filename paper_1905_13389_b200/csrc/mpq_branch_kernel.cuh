@@ -204,9 +204,13 @@ struct BranchLevel {
 
 template <int HB, int SB>
 struct BranchTile {
-    // k-quads whose xor words are compressed together: a 1 x 1 bit product has only 4 words per
-    // k-quad, too few for the adders to pay, so two k-quads are taken at once
-    static constexpr int GQ = (HB * SB == 1) ? 2 : 1;
+    // k-quads whose xor words are compressed together.  A product with a 1-bit operand has one plane
+    // pair per weight, i.e. only 4 xor words of equal weight per k-quad: a chain of adders over so few
+    // words leaves 3 of 4 (1 x 1) or 5 of 8 (1 x 2) population counts standing where half is the
+    // balance of the two pipes.  Two k-quads at once give every weight 8 words and the full budget of
+    // adders finds work (1 x 2 bits: 0.84 -> 0.90 of the instruction-mix peak).  From 1 x 3 bits on the
+    // gain (7 of 12 counts -> 6) no longer pays for the registers of a second k-quad.
+    static constexpr int GQ = (HB * SB <= 2) ? 2 : 1;
     static constexpr int TH = ((HB == 1) ? 8 : (HB == 2) ? 4 : (HB <= 4) ? 2 : 1) / GQ;   // TH*HB*GQ <= 8 quads held
     static constexpr int KQ = (SB == 1) ? 8 : (SB == 2) ? 4 : (SB <= 4) ? 2 : 1;   // k-quads per stage
     static constexpr int STAGES = 3;
