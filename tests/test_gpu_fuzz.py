@@ -184,3 +184,31 @@ def test_conv_encoded_random_cases(mpq, cuda, seed):
     assert np.array_equal(planes.cpu().numpy().view(np.uint32), want), key
     if keep:
         assert np.array_equal(yf.cpu().numpy(), ref), key
+
+
+@pytest.mark.parametrize("a_bits,w_bits,m,n,k", [
+    (2, 2, 64, 4090, 6144),      # 128 tiles of 32 columns, the last one 26 wide
+    (1, 1, 64, 4096, 12288),     # two k-quads per group
+    (4, 4, 64, 2044, 3200),      # two held tiles x 64
+    (8, 3, 33, 1000, 4096),      # 16-row held tiles, two k-groups
+    (2, 2, 64, 28, 6144),        # a single tile
+])
+def test_gemm_small_batch_k_group_shapes(mpq, cuda, a_bits, w_bits, m, n, k):
+    """Small-batch layers with at most one tile per multiprocessor (two or three k-groups per CTA):
+    ragged last tiles, every held-tile height, both outputs, glue in the store."""
+    x = inputs.uniform_levels(22, m + n, (m, k), a_bits)
+    w = inputs.uniform_levels(22, k, (n, k), w_bits)
+    acc_ref, out_ref, s_a, s_w = oracle.linear(x, w, a_bits, w_bits, w_per_row=True, a_act=oracle.HRELU)
+    bias = inputs.normal(22, 7, (n,))
+    want = oracle.epilogue(out_ref, bias, None, True)
+    xd, wd = _dev(x, cuda), _dev(w, cuda)
+    sa_d, sw_d = mpq.absmax(xd, 0, mpq.ACT_HRELU), mpq.absmax(wd, mpq.SCALE_PER_ROW)
+    ap, wp = mpq.encode(xd, sa_d, a_bits, 0, mpq.ACT_HRELU), mpq.encode(wd, sw_d, w_bits, mpq.SCALE_PER_ROW)
+    ci = torch.full((m, n), -5, dtype=torch.int32, device=cuda)
+    cf = torch.full((m, n), float("nan"), dtype=torch.float32, device=cuda)
+    mpq.gemm(ap, a_bits, wp, w_bits, m, n, k, ci, cf, sa_d, sw_d, mpq.SCALE_PER_ROW)
+    assert np.array_equal(ci.cpu().numpy(), acc_ref)
+    assert rel_close(cf.cpu().numpy(), out_ref)
+    cf.fill_(float("nan"))
+    mpq.gemm_fused(ap, a_bits, wp, w_bits, m, n, k, None, cf, sa_d, sw_d, mpq.SCALE_PER_ROW, _dev(bias, cuda), None, True)
+    assert rel_close(cf.cpu().numpy(), want)
