@@ -35,9 +35,9 @@ SIZE = 4096
 A_BITS = W_BITS = 2
 HBM_FALLBACK_GBS = 6650.0      # used only when MEASURED_PEAKS.json is absent
 # DRAM bytes per launch of the GEMM kernel (dram__bytes_read.sum + dram__bytes_write.sum) from the
-# kept ncu capture of this command: 8.48 MB + 79.9 MB.
+# kept ncu capture of this command: 8.46 MB + 79.54 MB.
 # Set back to None whenever branch_kernel changes after that capture.
-GEMM_DRAM_TRAFFIC_BYTES = 88.4e6
+GEMM_DRAM_TRAFFIC_BYTES = 88.0e6
 ORACLE_SAMPLE_ROWS = 1024      # activation rows of the bounded sample the CPU oracle is timed on
 
 
@@ -465,7 +465,8 @@ def run_cuda(args):
                                          "ms_per_step": e2e_prepared_ms / e2e_steps, "h2d_bytes_per_step": m * k * 4,
                                          "d2h_bytes_per_step": 2 * m * n * 4,
                                          "api": "mpq_linear_host_prepared (weights encoded once, resident on the device)"}},
-            "gpu_launches": 5 * args.steps,
+            # per step: 2 x (zeroing kernel + range kernel), 2 x encoder, 1 x branch GEMM
+            "gpu_launches": 7 * args.steps,
             "clocks": clocks.summary(),
         }
         suite = None
