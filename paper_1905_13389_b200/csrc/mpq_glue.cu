@@ -103,6 +103,10 @@ stem_conv7x7_kernel(const float* __restrict__ x, const float* __restrict__ w, fl
 // 3x3 max-pool, stride 2, pad 1 (padding never wins: the window always holds a real element).
 // A thread produces four adjacent outputs of a row from the 3 x 9 inputs they share, so that
 // 27 loads are in flight per thread and neighbouring threads read neighbouring columns.
+// VEC: W is a multiple of 8 and x is 16-byte aligned -- the eight inputs 8g .. 8g+7 of a group are
+// two aligned 16-byte loads, and the ninth (8g - 1) is the left neighbour's last element, taken
+// from the neighbouring lane when that lane holds the same row's previous group.
+template <bool VEC>
 __global__ void maxpool3x3s2_kernel(const float* __restrict__ x, float* __restrict__ y,
                                     int64_t planes, int H, int W, int Ho, int Wo, float* out_max) {
     chain_entry();
@@ -111,6 +115,8 @@ __global__ void maxpool3x3s2_kernel(const float* __restrict__ x, float* __restri
     const int64_t total = planes * Ho * groups;
     const int64_t stride = (int64_t)gridDim.x * blockDim.x;
     const float ninf = -__int_as_float(0x7f800000);
+    // (VEC: every lane of a warp runs the same number of iterations up to the last one, where the
+    // shuffle below names the lanes that are still in the loop)
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += stride) {
         const int g = (int)(i % groups), oh = (int)((i / groups) % Ho);
         const int64_t pl = i / ((int64_t)groups * Ho);
@@ -119,15 +125,49 @@ __global__ void maxpool3x3s2_kernel(const float* __restrict__ x, float* __restri
         float col[9];                                      // column maxima over the three rows
 #pragma unroll
         for (int q = 0; q < 9; ++q) col[q] = ninf;
+        if (VEC) {
+            const unsigned live = __activemask();
+            float4 lo[3], hi[3];
 #pragma unroll
-        for (int kh = 0; kh < 3; ++kh) {
-            const int ih = 2 * oh + kh - 1;
-            if (ih < 0 || ih >= H) continue;
-            const float* row = xp + (int64_t)ih * W;
+            for (int kh = 0; kh < 3; ++kh) {
+                const int ih = 2 * oh + kh - 1;
+                const bool in = ih >= 0 && ih < H;
+                const float4* row = reinterpret_cast<const float4*>(xp + (int64_t)(in ? ih : 0) * W + 8 * g);
+                lo[kh] = in ? __ldg(row) : make_float4(ninf, ninf, ninf, ninf);
+                hi[kh] = in ? __ldg(row + 1) : make_float4(ninf, ninf, ninf, ninf);
+            }
 #pragma unroll
-            for (int q = 0; q < 9; ++q) {
-                const int iw = iw0 + q;
-                if (iw >= 0 && iw < W) col[q] = fmaxf(col[q], __ldg(row + iw));
+            for (int kh = 0; kh < 3; ++kh) {
+                col[1] = fmaxf(col[1], lo[kh].x); col[2] = fmaxf(col[2], lo[kh].y);
+                col[3] = fmaxf(col[3], lo[kh].z); col[4] = fmaxf(col[4], lo[kh].w);
+                col[5] = fmaxf(col[5], hi[kh].x); col[6] = fmaxf(col[6], hi[kh].y);
+                col[7] = fmaxf(col[7], hi[kh].z); col[8] = fmaxf(col[8], hi[kh].w);
+            }
+            // column 8g - 1: the left neighbour's column 8(g-1) + 7, already reduced over the three rows
+            const float left = __shfl_up_sync(live, col[8], 1);
+            const int lane = (int)(threadIdx.x & 31);
+            if (g > 0) {
+                if (lane > 0 && ((live >> (lane - 1)) & 1u)) {
+                    col[0] = left;                         // lane - 1 holds item i - 1: same row, group g - 1
+                } else {
+#pragma unroll
+                    for (int kh = 0; kh < 3; ++kh) {
+                        const int ih = 2 * oh + kh - 1;
+                        if (ih >= 0 && ih < H) col[0] = fmaxf(col[0], __ldg(xp + (int64_t)ih * W + iw0));
+                    }
+                }
+            }
+        } else {
+#pragma unroll
+            for (int kh = 0; kh < 3; ++kh) {
+                const int ih = 2 * oh + kh - 1;
+                if (ih < 0 || ih >= H) continue;
+                const float* row = xp + (int64_t)ih * W;
+#pragma unroll
+                for (int q = 0; q < 9; ++q) {
+                    const int iw = iw0 + q;
+                    if (iw >= 0 && iw < W) col[q] = fmaxf(col[q], __ldg(row + iw));
+                }
             }
         }
         float* dst = y + (pl * Ho + oh) * Wo + ow0;
@@ -174,8 +214,9 @@ extern "C" int mpq_maxpool3x3s2(const float* x, float* y, int N, int C, int H, i
     const int sms = sm_count();
     if (sms <= 0) return MPQ_ERR_CUDA;
     const int64_t blocks = min((int64_t)sms * 32, ceil_div(total, 256));
-    return launch_chained(maxpool3x3s2_kernel, (unsigned)blocks, 256, 0, (cudaStream_t)stream,
-                          x, y, (int64_t)N * C, H, W, Ho, Wo, out_max);
+    const bool vec = W % 8 == 0 && aligned16(x);
+    return launch_chained(vec ? maxpool3x3s2_kernel<true> : maxpool3x3s2_kernel<false>, (unsigned)blocks, 256, 0,
+                          (cudaStream_t)stream, x, y, (int64_t)N * C, H, W, Ho, Wo, out_max);
 }
 
 extern "C" int mpq_zero(void* p, int64_t bytes, void* stream) {
