@@ -20,7 +20,7 @@ constexpr int kStemCols = 4 * kStemGroups;          // 56
 constexpr int kStemThreads = kStemRows * kStemGroups;   // 224
 constexpr int kStemPatchH = 2 * kStemRows + 5;      // 37
 constexpr int kStemPatchW = 2 * kStemCols + 5;      // 117
-constexpr int kStemPatchStride = kStemPatchW + 1;   // 118
+constexpr int kStemPatchStride = 120;               // >= 117, rows 16-byte aligned: a thread's 13 inputs are three vector loads + one
 constexpr int kStemTaps = 3 * 7 * 7;                // 147
 constexpr int kStemO = 64;
 constexpr int kStemWRow = 68;                      // floats per staged weight row (64 + 4: spreads the transposing stores over banks)
@@ -31,7 +31,7 @@ stem_conv7x7_kernel(const float* __restrict__ x, const float* __restrict__ w, fl
     extern __shared__ __align__(16) float smem[];
     chain_entry();
     float* ws = smem;                                   // [147][68]
-    float* xs = smem + kStemTaps * kStemWRow;           // [3][37][118]
+    float* xs = smem + kStemTaps * kStemWRow;           // [3][37][120]
     const int tid = threadIdx.x;
     const int tiles_w = (Wo + kStemCols - 1) / kStemCols;
     const int tiles_h = (Ho + kStemRows - 1) / kStemRows;
@@ -67,8 +67,14 @@ stem_conv7x7_kernel(const float* __restrict__ x, const float* __restrict__ w, fl
             for (int kh = 0; kh < 7; ++kh) {
                 const float* xrow = xs + (c * kStemPatchH + 2 * ty + kh) * kStemPatchStride + 8 * tg;
                 float xv[13];
-#pragma unroll
-                for (int q = 0; q < 13; ++q) xv[q] = xrow[q];
+                {
+                    const float4* xq = reinterpret_cast<const float4*>(xrow);     // 8 * tg floats into an aligned row
+                    const float4 a = xq[0], b = xq[1], d = xq[2];
+                    xv[0] = a.x; xv[1] = a.y; xv[2] = a.z; xv[3] = a.w;
+                    xv[4] = b.x; xv[5] = b.y; xv[6] = b.z; xv[7] = b.w;
+                    xv[8] = d.x; xv[9] = d.y; xv[10] = d.z; xv[11] = d.w;
+                    xv[12] = xrow[12];
+                }
                 const float* wrow = ws + ((c * 7 + kh) * 7) * kStemWRow + o0;
 #pragma unroll
                 for (int kw = 0; kw < 7; ++kw) {
