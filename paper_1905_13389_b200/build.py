@@ -21,7 +21,7 @@ FLAGS = ["-O3", "-std=c++17", "-lineinfo", "-Xcompiler", "-fPIC", "-I", INCLUDE,
 # IEEE arithmetic is part of the contract (bit-exact codes): never --use_fast_math / -ftz.
 
 PLAIN = ["mpq_api.cu", "mpq_encode.cu", "mpq_encode_trig.cu", "mpq_gemm.cu", "mpq_glue.cu", "mpq_probe.cu"]
-HEADERS = ["mpq_common.cuh", "mpq_branch_kernel.cuh", "mpq_branch_launch.cuh", os.path.join(INCLUDE, "mpq.h")]
+HEADERS = ["mpq_common.cuh", "mpq_branch_kernel.cuh", "mpq_branch_launch.cuh", "mpq_pointwise_kernel.cuh", os.path.join(INCLUDE, "mpq.h")]
 
 
 def _jobs():

@@ -1,5 +1,6 @@
 // C-ABI entry points of the layer product: argument checks, then dispatch on the bit-widths.
 #include "mpq_branch_launch.cuh"
+#include "mpq_pointwise_kernel.cuh"
 
 namespace mpq {
 
@@ -30,6 +31,20 @@ static int dispatch_conv(int hb, int sb, const BranchParams& p, cudaStream_t st)
         case 6: return launch_conv_hb<6>(sb, p, st);
         case 7: return launch_conv_hb<7>(sb, p, st);
         case 8: return launch_conv_hb<8>(sb, p, st);
+    }
+    return MPQ_ERR_UNSUPPORTED;
+}
+
+static int dispatch_pointwise(int hb, int sb, const BranchParams& p, cudaStream_t st) {
+    switch (hb) {
+        case 1: return launch_pointwise_hb<1>(sb, p, st);
+        case 2: return launch_pointwise_hb<2>(sb, p, st);
+        case 3: return launch_pointwise_hb<3>(sb, p, st);
+        case 4: return launch_pointwise_hb<4>(sb, p, st);
+        case 5: return launch_pointwise_hb<5>(sb, p, st);
+        case 6: return launch_pointwise_hb<6>(sb, p, st);
+        case 7: return launch_pointwise_hb<7>(sb, p, st);
+        case 8: return launch_pointwise_hb<8>(sb, p, st);
     }
     return MPQ_ERR_UNSUPPORTED;
 }
@@ -174,6 +189,7 @@ extern "C" int mpq_conv_encoded(const uint32_t* x_planes, int a_bits, int N, int
     p.out_h0 = 0; p.out_w0 = 0; p.out_step = 1;
     p.window3x3 = KH == 3 ? 1 : 0;
     // held = weights (w_bits planes), streamed = activations (a_bits planes)
+    if (pointwise_applies(p)) return dispatch_pointwise(w_bits, a_bits, p, (cudaStream_t)stream);
     return dispatch_conv(w_bits, a_bits, p, (cudaStream_t)stream);
 }
 

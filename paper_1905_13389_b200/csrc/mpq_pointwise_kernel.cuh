@@ -1,0 +1,132 @@
+// 1 x 1 convolution over few channels (C <= 256, no padding): the pixel-stationary form of the
+// branch-fused product.
+//
+// With k = C of at most 8 words a tile of the general kernel has a single, partly filled k-stage and
+// its per-tile set-up outweighs the branch arithmetic (a 64-channel shortcut convolution ran at 0.46
+// of the instruction-mix peak).  Here a thread owns ONE output pixel: it reads that pixel's SB x C/32
+// plane words once, keeps them in registers, and walks over the output channels of its CTA, whose
+// weight planes sit in shared memory and are read as broadcasts.  No staging ring, no k-loop, no
+// barrier after the set-up; per output there are only the branch arithmetic (the same carry-save
+// levels as the general kernel), HB x NQ shared-memory loads and the store.
+//
+// Grid: x = blocks of 256 output pixels, y = blocks of kPointwiseChannels output channels.
+// NQ = 16-byte chunks per pixel and plane (1: C <= 128, 2: C = 256); NW = words of a chunk that hold
+// data (2 for C = 32 / 64, whose chunk is zero-filled, else 4).
+#pragma once
+#include "mpq_branch_kernel.cuh"
+
+namespace mpq {
+
+constexpr int kPointwiseChannels = 32;
+
+template <int HB, int SB, int NQ, int NW>
+__global__ void __launch_bounds__(256)
+pointwise_kernel(const BranchParams p) {
+    __shared__ uint4 wq[kPointwiseChannels * HB * NQ];      // [channel][plane][chunk]
+    __shared__ float alpha_s[kPointwiseChannels];
+    chain_entry();
+    const int tid = (int)threadIdx.x;
+    const int o_base = (int)blockIdx.y * kPointwiseChannels;
+    const int oc = min(kPointwiseChannels, p.O - o_base);
+    const bool want_f32 = p.out_f32 != nullptr;
+    // weights of this CTA's channels: rows are zero-padded to whole 16-byte chunks
+    for (int i = tid; i < oc * HB * NQ; i += 256) {
+        const int q = i % NQ, plane = (i / NQ) % HB, o = i / (NQ * HB);
+        wq[i] = __ldg(reinterpret_cast<const uint4*>(p.held + ((int64_t)plane * p.held_plane_rows + o_base + o) * p.rw) + q);
+    }
+    if (tid < oc && want_f32) {
+        const float fa = __fdiv_rn(__ldg(p.a_scale), (float)((1 << SB) - 1));
+        alpha_s[tid] = __fmul_rn(fa, __fdiv_rn(__ldg(p.w_scale + (p.w_per_row ? o_base + tid : 0)), (float)((1 << HB) - 1)));
+    }
+    __syncthreads();
+
+    const int64_t g = (int64_t)blockIdx.x * 256 + tid;      // output pixel (n, oh, ow)
+    const int64_t hw = (int64_t)p.Ho * p.Wo;
+    float seen_max = 0.0f;
+    if (g < p.streamed_rows) {
+        const int n = (int)(g / hw);
+        const int rem = (int)(g % hw);
+        const int64_t pix = ((int64_t)n * p.H + (rem / p.Wo) * p.stride) * p.W + (rem % p.Wo) * p.stride;
+        const int64_t plane_words = (int64_t)p.N * p.H * p.W * p.Cw;
+        uint4 s[NQ][SB];
+#pragma unroll
+        for (int j = 0; j < SB; ++j) {
+            const uint32_t* src = p.streamed + j * plane_words + pix * p.Cw;
+            if (NQ == 2) {
+                s[0][j] = __ldg(reinterpret_cast<const uint4*>(src));
+                s[NQ - 1][j] = __ldg(reinterpret_cast<const uint4*>(src) + 1);
+            } else if (NW == 4) {
+                s[0][j] = __ldg(reinterpret_cast<const uint4*>(src));
+            } else if (p.Cw == 2) {
+                const uint2 v = __ldg(reinterpret_cast<const uint2*>(src));
+                s[0][j] = make_uint4(v.x, v.y, 0u, 0u);
+            } else {
+                s[0][j] = make_uint4(__ldg(src), 0u, 0u, 0u);
+            }
+        }
+        constexpr uint32_t LL = (uint32_t)(((1 << HB) - 1) * ((1 << SB) - 1));
+        const uint32_t full = LL * (uint32_t)p.k;
+        const uint32_t none[1] = {0u};
+        const int64_t out0 = ((int64_t)n * p.O + o_base) * hw + rem;
+#pragma unroll 1
+        for (int o = 0; o < oc; ++o) {
+            uint32_t acc = 0u;
+#pragma unroll
+            for (int q = 0; q < NQ; ++q) {
+                uint4 h[HB];
+#pragma unroll
+                for (int i = 0; i < HB; ++i) h[i] = wq[(o * HB + i) * NQ + q];
+                BranchLevel<HB, SB, 1, NW, 0, 0, (2 * HB * SB * NW) / 4>::run(h, s[q], none, acc, p);
+            }
+            const int32_t v = (int32_t)(full - 2u * acc);
+            const int64_t idx = out0 + (int64_t)o * hw;
+            if (p.out_i32) p.out_i32[idx] = v;
+            if (want_f32) {
+                float f = __fmul_rn((float)v, alpha_s[o]);
+                if (p.residual) f = __fadd_rn(f, __ldg(p.residual + idx));
+                if (p.relu) f = fmaxf(f, 0.0f);
+                p.out_f32[idx] = f;
+                seen_max = fmaxf(seen_max, f);
+            }
+        }
+    }
+    if (p.out_max) {
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) seen_max = fmaxf(seen_max, __shfl_xor_sync(0xffffffffu, seen_max, off));
+        if ((tid & 31) == 0 && seen_max > 0.0f) atomicMax(reinterpret_cast<int*>(p.out_max), __float_as_int(seen_max));
+    }
+}
+
+// Takes the layers that mpq_conv would otherwise run as tiles with a single k-stage.
+inline bool pointwise_applies(const BranchParams& p) {
+    return p.KH == 1 && p.KW == 1 && p.pad == 0 && p.Cw <= 8 && p.next_planes == nullptr;
+}
+
+template <int HB, int SB>
+static int launch_pointwise(const BranchParams& p, cudaStream_t st) {
+    const int64_t bx = ceil_div(p.streamed_rows, 256), by = ceil_div(p.O, kPointwiseChannels);
+    if (bx <= 0 || bx > 0x7fffffffLL || by > 65535) return MPQ_ERR_BAD_SHAPE;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)bx, (unsigned)by, 1);
+    cfg.blockDim = dim3(256, 1, 1);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = bx * by >= 1024 ? 1 : 0;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaError_t e;
+    if (p.Cw == 8) e = cudaLaunchKernelEx(&cfg, pointwise_kernel<HB, SB, 2, 4>, p);
+    else if (p.Cw == 4) e = cudaLaunchKernelEx(&cfg, pointwise_kernel<HB, SB, 1, 4>, p);
+    else e = cudaLaunchKernelEx(&cfg, pointwise_kernel<HB, SB, 1, 2>, p);
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        return MPQ_ERR_CUDA;
+    }
+    return launch_status();
+}
+
+template <int HB>
+int launch_pointwise_hb(int sb, const BranchParams& p, cudaStream_t st);
+
+}  // namespace mpq

@@ -212,3 +212,37 @@ def test_gemm_small_batch_k_group_shapes(mpq, cuda, a_bits, w_bits, m, n, k):
     cf.fill_(float("nan"))
     mpq.gemm_fused(ap, a_bits, wp, w_bits, m, n, k, None, cf, sa_d, sw_d, mpq.SCALE_PER_ROW, _dev(bias, cuda), None, True)
     assert rel_close(cf.cpu().numpy(), want)
+
+
+@pytest.mark.parametrize("C", [32, 64, 128, 256])
+@pytest.mark.parametrize("a_bits,w_bits,stride", [(4, 4, 2), (1, 1, 1), (8, 8, 2), (3, 5, 1), (2, 7, 2)])
+def test_pointwise_conv_small_channel_counts(mpq, cuda, C, a_bits, w_bits, stride):
+    """1 x 1 convolutions over at most 256 channels (the shortcut convolutions of a residual stack): one
+    thread per output pixel, output channels in blocks of 32.  Ragged pixel and channel counts, both
+    outputs, residual + max(., 0) + the next encoder's range in the store; per-tensor weight range too."""
+    N, H, W, O = 3, 13, 11, 72                        # 3 * 7 * 6 = 126 or 429 pixels, 72 = 2 * 32 + 8 channels
+    if a_bits + w_bits > 12:
+        O = 40
+    x = inputs.uniform_levels(24, C + stride, (N, C, H, W), a_bits)
+    w = inputs.uniform_levels(24, 100 + C, (O, C, 1, 1), w_bits) * np.float32(0.37)
+    for per_channel in (True, False):
+        acc_ref, out_ref, s_a, s_w = oracle.conv_layer(x, w, a_bits, w_bits, stride, 0, per_channel, oracle.HRELU)
+        res = inputs.normal(24, 7, out_ref.shape)
+        want = oracle.epilogue(out_ref, None, res, True)
+        xd, wd = _dev(x, cuda), _dev(w, cuda)
+        mode = mpq.SCALE_PER_ROW if per_channel else mpq.SCALE_PER_TENSOR
+        sa_d, sw_d = mpq.absmax(xd, 0, mpq.ACT_HRELU), mpq.absmax(wd, mode)
+        xp = mpq.encode_nchw(xd, sa_d, a_bits, mpq.ACT_HRELU)
+        wp, taps = mpq.encode_oihw(wd, sw_d, w_bits, mode)
+        yi = torch.full(acc_ref.shape, -5, dtype=torch.int32, device=cuda)
+        yf = torch.full(acc_ref.shape, float("nan"), dtype=torch.float32, device=cuda)
+        mpq.conv(xp, a_bits, N, C, H, W, wp, w_bits, taps, O, 1, 1, stride, 0, yi, yf, sa_d, sw_d, mode)
+        assert np.array_equal(yi.cpu().numpy(), acc_ref)
+        assert rel_close(yf.cpu().numpy(), out_ref)
+        out_max = torch.zeros(1, dtype=torch.float32, device=cuda)
+        yf.fill_(float("nan"))
+        mpq.conv_fused(xp, a_bits, N, C, H, W, wp, w_bits, taps, O, 1, 1, stride, 0, None, yf, sa_d, sw_d, mode,
+                       _dev(res, cuda), True, out_max)
+        got = yf.cpu().numpy()
+        assert rel_close(got, want)
+        assert float(out_max.item()) == float(got.max())
