@@ -54,4 +54,15 @@ int launch_pointwise_hb<MPQ_HB>(int sb, const BranchParams& p, cudaStream_t st) 
     return MPQ_ERR_UNSUPPORTED;
 }
 
+template <>
+int launch_window3x3c64_hb<MPQ_HB>(int sb, const BranchParams& p, cudaStream_t st) {
+    switch (sb) {
+        case 1: return launch_window3x3c64<MPQ_HB, 1>(p, st);
+        case 2: return launch_window3x3c64<MPQ_HB, 2>(p, st);
+        case 3: return launch_window3x3c64<MPQ_HB, 3>(p, st);
+        case 4: return launch_window3x3c64<MPQ_HB, 4>(p, st);
+    }
+    return MPQ_ERR_UNSUPPORTED;
+}
+
 }  // namespace mpq

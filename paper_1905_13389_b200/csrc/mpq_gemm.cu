@@ -49,6 +49,20 @@ static int dispatch_pointwise(int hb, int sb, const BranchParams& p, cudaStream_
     return MPQ_ERR_UNSUPPORTED;
 }
 
+static int dispatch_window3x3c64(int hb, int sb, const BranchParams& p, cudaStream_t st) {
+    switch (hb) {
+        case 1: return launch_window3x3c64_hb<1>(sb, p, st);
+        case 2: return launch_window3x3c64_hb<2>(sb, p, st);
+        case 3: return launch_window3x3c64_hb<3>(sb, p, st);
+        case 4: return launch_window3x3c64_hb<4>(sb, p, st);
+        case 5: return launch_window3x3c64_hb<5>(sb, p, st);
+        case 6: return launch_window3x3c64_hb<6>(sb, p, st);
+        case 7: return launch_window3x3c64_hb<7>(sb, p, st);
+        case 8: return launch_window3x3c64_hb<8>(sb, p, st);
+    }
+    return MPQ_ERR_UNSUPPORTED;
+}
+
 static void fill_pow2(BranchParams& p) {
     for (int e = 0; e < 24; ++e) p.pow2[e] = 1u << e;
 }
@@ -190,6 +204,7 @@ extern "C" int mpq_conv_encoded(const uint32_t* x_planes, int a_bits, int N, int
     p.window3x3 = KH == 3 ? 1 : 0;
     // held = weights (w_bits planes), streamed = activations (a_bits planes)
     if (pointwise_applies(p)) return dispatch_pointwise(w_bits, a_bits, p, (cudaStream_t)stream);
+    if (window3x3c64_applies(p, a_bits)) return dispatch_window3x3c64(w_bits, a_bits, p, (cudaStream_t)stream);
     return dispatch_conv(w_bits, a_bits, p, (cudaStream_t)stream);
 }
 

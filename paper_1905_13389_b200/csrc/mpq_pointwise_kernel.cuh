@@ -97,6 +97,134 @@ pointwise_kernel(const BranchParams p) {
     }
 }
 
+// ------------------------------------------------------------------------------------------
+// 3 x 3 convolution over 64 channels, pixel-stationary.  k = 576 is 18 words: the general kernel's
+// tile runs two and a quarter k-stages and pays its set-up, ring and gather for them (0.82 of the
+// instruction-mix peak).  A thread keeps the 9 taps x 2 words x SB planes of its output pixel in
+// registers (taps outside the image as zero bits, i.e. as the code -L_a, taken out again through the
+// tap sums exactly as in the general kernel) and walks over up to 64 output channels whose weight
+// rows -- five 16-byte chunks per plane, the last one half filled -- are broadcast from shared memory.
+// ------------------------------------------------------------------------------------------
+constexpr int kWindowChannels = 64;
+
+template <int HB, int SB>
+__global__ void __launch_bounds__(256)
+window3x3c64_kernel(const BranchParams p) {
+    constexpr int NQ = 5;                                    // 18 words = four chunks and a half
+    __shared__ uint4 wq[kWindowChannels * HB * NQ];          // [channel][plane][chunk]
+    __shared__ float alpha_s[kWindowChannels];
+    __shared__ int tap_s[9 * kWindowChannels];               // [tap][channel]
+    chain_entry();
+    const int tid = (int)threadIdx.x;
+    const int o_base = (int)blockIdx.y * kWindowChannels;
+    const int oc = min(kWindowChannels, p.O - o_base);
+    const bool want_f32 = p.out_f32 != nullptr;
+    for (int i = tid; i < oc * HB * NQ; i += 256) {
+        const int q = i % NQ, plane = (i / NQ) % HB, o = i / (NQ * HB);
+        wq[i] = __ldg(reinterpret_cast<const uint4*>(p.held + ((int64_t)plane * p.held_plane_rows + o_base + o) * p.rw) + q);
+    }
+    if (p.tap_sums)
+        for (int i = tid; i < 9 * oc; i += 256) tap_s[(i / oc) * kWindowChannels + i % oc] = __ldg(p.tap_sums + (int64_t)(i / oc) * p.O + o_base + i % oc);
+    if (tid < oc && want_f32) {
+        const float fa = __fdiv_rn(__ldg(p.a_scale), (float)((1 << SB) - 1));
+        alpha_s[tid] = __fmul_rn(fa, __fdiv_rn(__ldg(p.w_scale + (p.w_per_row ? o_base + tid : 0)), (float)((1 << HB) - 1)));
+    }
+    __syncthreads();
+
+    const int64_t g = (int64_t)blockIdx.x * 256 + tid;      // output pixel (n, oh, ow)
+    const int64_t hw = (int64_t)p.Ho * p.Wo;
+    float seen_max = 0.0f;
+    if (g < p.streamed_rows) {
+        const int n = (int)(g / hw);
+        const int rem = (int)(g % hw);
+        const int ih0 = (rem / p.Wo) * p.stride - p.pad, iw0 = (rem % p.Wo) * p.stride - p.pad;
+        const int64_t plane_words = (int64_t)p.N * p.H * p.W * 2;
+        uint4 s[NQ][SB];
+        unsigned outside = 0u;
+#pragma unroll
+        for (int t = 0; t < 9; ++t) {
+            const int ih = ih0 + t / 3, iw = iw0 + t % 3;
+            const bool in = ih >= 0 && ih < p.H && iw >= 0 && iw < p.W;
+            if (!in) outside |= 1u << t;
+            const uint32_t* src = p.streamed + (in ? (((int64_t)n * p.H + ih) * p.W + iw) * 2 : 0);
+#pragma unroll
+            for (int j = 0; j < SB; ++j) {
+                const uint2 v = in ? __ldg(reinterpret_cast<const uint2*>(src + j * plane_words)) : make_uint2(0u, 0u);
+                if (t % 2 == 0) { s[t / 2][j].x = v.x; s[t / 2][j].y = v.y; }
+                else { s[t / 2][j].z = v.x; s[t / 2][j].w = v.y; }
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < SB; ++j) { s[NQ - 1][j].z = 0u; s[NQ - 1][j].w = 0u; }
+        constexpr uint32_t LL = (uint32_t)(((1 << HB) - 1) * ((1 << SB) - 1));
+        const uint32_t full = LL * (uint32_t)p.k;
+        const uint32_t none[1] = {0u};
+        const int64_t out0 = ((int64_t)n * p.O + o_base) * hw + rem;
+#pragma unroll 1
+        for (int o = 0; o < oc; ++o) {
+            uint32_t acc = 0u;
+#pragma unroll
+            for (int q = 0; q < NQ; ++q) {
+                uint4 h[HB];
+#pragma unroll
+                for (int i = 0; i < HB; ++i) h[i] = wq[(o * HB + i) * NQ + q];
+                if (q < NQ - 1) BranchLevel<HB, SB, 1, 4, 0, 0, 2 * HB * SB>::run(h, s[q], none, acc, p);
+                else BranchLevel<HB, SB, 1, 2, 0, 0, HB * SB>::run(h, s[q], none, acc, p);
+            }
+            int32_t v = (int32_t)(full - 2u * acc);
+            if (outside) {
+                uint32_t fix = 0u;
+                for (int t = 0; t < 9; ++t)
+                    if (outside & (1u << t)) fix += (uint32_t)tap_s[t * kWindowChannels + o];
+                v = (int32_t)((uint32_t)v + (uint32_t)((1 << SB) - 1) * fix);
+            }
+            const int64_t idx = out0 + (int64_t)o * hw;
+            if (p.out_i32) p.out_i32[idx] = v;
+            if (want_f32) {
+                float f = __fmul_rn((float)v, alpha_s[o]);
+                if (p.residual) f = __fadd_rn(f, __ldg(p.residual + idx));
+                if (p.relu) f = fmaxf(f, 0.0f);
+                p.out_f32[idx] = f;
+                seen_max = fmaxf(seen_max, f);
+            }
+        }
+    }
+    if (p.out_max) {
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) seen_max = fmaxf(seen_max, __shfl_xor_sync(0xffffffffu, seen_max, off));
+        if ((tid & 31) == 0 && seen_max > 0.0f) atomicMax(reinterpret_cast<int*>(p.out_max), __float_as_int(seen_max));
+    }
+}
+
+// (activations of up to 4 bits: 18 words per plane must stay in registers)
+inline bool window3x3c64_applies(const BranchParams& p, int a_bits) {
+    return p.KH == 3 && p.KW == 3 && p.Cw == 2 && a_bits <= 4 && p.next_planes == nullptr &&
+           (p.pad == 0 || p.tap_sums != nullptr);
+}
+
+template <int HB, int SB>
+static int launch_window3x3c64(const BranchParams& p, cudaStream_t st) {
+    const int64_t bx = ceil_div(p.streamed_rows, 256), by = ceil_div(p.O, kWindowChannels);
+    if (bx <= 0 || bx > 0x7fffffffLL || by > 65535) return MPQ_ERR_BAD_SHAPE;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)bx, (unsigned)by, 1);
+    cfg.blockDim = dim3(256, 1, 1);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = bx * by >= 1024 ? 1 : 0;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, window3x3c64_kernel<HB, SB>, p) != cudaSuccess) {
+        cudaGetLastError();
+        return MPQ_ERR_CUDA;
+    }
+    return launch_status();
+}
+
+template <int HB>
+int launch_window3x3c64_hb(int sb, const BranchParams& p, cudaStream_t st);
+
 // Takes the layers that mpq_conv would otherwise run as tiles with a single k-stage.
 inline bool pointwise_applies(const BranchParams& p) {
     return p.KH == 1 && p.KW == 1 && p.pad == 0 && p.Cw <= 8 && p.next_planes == nullptr;

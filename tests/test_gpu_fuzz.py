@@ -246,3 +246,36 @@ def test_pointwise_conv_small_channel_counts(mpq, cuda, C, a_bits, w_bits, strid
         got = yf.cpu().numpy()
         assert rel_close(got, want)
         assert float(out_max.item()) == float(got.max())
+
+
+@pytest.mark.parametrize("stride,pad", [(1, 1), (2, 1), (1, 0), (2, 0)])
+@pytest.mark.parametrize("a_bits,w_bits", [(4, 4), (1, 8), (3, 2), (2, 5), (5, 4)])
+def test_conv3x3_over_64_channels(mpq, cuda, a_bits, w_bits, stride, pad):
+    """3 x 3 convolutions over 64 channels (the first stage of a residual stack): with activations of up to
+    4 bits one thread keeps the whole window of its output pixel in registers; 5 bits take the tiled kernel.
+    Small images (every pixel on the border at 3 x 4), ragged pixel and channel counts, both outputs,
+    residual + max(., 0) + the next encoder's range in the store."""
+    for (N, H, W, O) in ((2, 3, 4, 8), (3, 12, 9, 72)):
+        if a_bits + w_bits > 8:
+            O = min(O, 40)
+        x = inputs.uniform_levels(25, 10 * stride + pad, (N, 64, H, W), a_bits)
+        w = inputs.uniform_levels(25, 50 + O, (O, 64, 3, 3), w_bits) * np.float32(1.7)
+        acc_ref, out_ref, s_a, s_w = oracle.conv_layer(x, w, a_bits, w_bits, stride, pad, True, oracle.HRELU)
+        res = inputs.normal(25, 7, out_ref.shape)
+        want = oracle.epilogue(out_ref, None, res, True)
+        xd, wd = _dev(x, cuda), _dev(w, cuda)
+        sa_d, sw_d = mpq.absmax(xd, 0, mpq.ACT_HRELU), mpq.absmax(wd, mpq.SCALE_PER_ROW)
+        xp = mpq.encode_nchw(xd, sa_d, a_bits, mpq.ACT_HRELU)
+        wp, taps = mpq.encode_oihw(wd, sw_d, w_bits, mpq.SCALE_PER_ROW)
+        yi = torch.full(acc_ref.shape, -5, dtype=torch.int32, device=cuda)
+        yf = torch.full(acc_ref.shape, float("nan"), dtype=torch.float32, device=cuda)
+        mpq.conv(xp, a_bits, N, 64, H, W, wp, w_bits, taps, O, 3, 3, stride, pad, yi, yf, sa_d, sw_d, mpq.SCALE_PER_ROW)
+        assert np.array_equal(yi.cpu().numpy(), acc_ref), (N, H, W, O)
+        assert rel_close(yf.cpu().numpy(), out_ref), (N, H, W, O)
+        out_max = torch.zeros(1, dtype=torch.float32, device=cuda)
+        yf.fill_(float("nan"))
+        mpq.conv_fused(xp, a_bits, N, 64, H, W, wp, w_bits, taps, O, 3, 3, stride, pad, None, yf, sa_d, sw_d,
+                       mpq.SCALE_PER_ROW, _dev(res, cuda), True, out_max)
+        got = yf.cpu().numpy()
+        assert rel_close(got, want), (N, H, W, O)
+        assert float(out_max.item()) == float(got.max())
