@@ -107,18 +107,25 @@ pointwise_kernel(const BranchParams p) {
 // ------------------------------------------------------------------------------------------
 constexpr int kWindowChannels = 64;
 
-template <int HB, int SB>
+// PLANES: the store also runs the consumer's Encoder (a variant of its own: the plain store keeps
+// its registers).
+template <int HB, int SB, bool PLANES>
 __global__ void __launch_bounds__(256)
 window3x3c64_kernel(const BranchParams p) {
     constexpr int NQ = 5;                                    // 18 words = four chunks and a half
-    __shared__ uint4 wq[kWindowChannels * HB * NQ];          // [channel][plane][chunk]
-    __shared__ float alpha_s[kWindowChannels];
-    __shared__ int tap_s[9 * kWindowChannels];               // [tap][channel]
+    extern __shared__ uint4 window_smem[];
+    uint4* wq = window_smem;                                 // [channel][plane][chunk]
+    float* alpha_s = reinterpret_cast<float*>(wq + kWindowChannels * HB * NQ);
+    int* tap_s = reinterpret_cast<int*>(alpha_s + kWindowChannels);          // [tap][channel]
+    // consumer's Encoder in the store: level indices [channel][thread], one byte each (16 KB); a thread
+    // reads back only its own column, so no barrier is needed
+    unsigned char* code_s = reinterpret_cast<unsigned char*>(tap_s + 9 * kWindowChannels);
     chain_entry();
     const int tid = (int)threadIdx.x;
     const int o_base = (int)blockIdx.y * kWindowChannels;
     const int oc = min(kWindowChannels, p.O - o_base);
-    const bool want_f32 = p.out_f32 != nullptr;
+    constexpr bool want_planes = PLANES;
+    const bool want_f32 = p.out_f32 != nullptr || want_planes;
     for (int i = tid; i < oc * HB * NQ; i += 256) {
         const int q = i % NQ, plane = (i / NQ) % HB, o = i / (NQ * HB);
         wq[i] = __ldg(reinterpret_cast<const uint4*>(p.held + ((int64_t)plane * p.held_plane_rows + o_base + o) * p.rw) + q);
@@ -160,6 +167,14 @@ window3x3c64_kernel(const BranchParams p) {
         const uint32_t full = LL * (uint32_t)p.k;
         const uint32_t none[1] = {0u};
         const int64_t out0 = ((int64_t)n * p.O + o_base) * hw + rem;
+        float next_inv = 0.0f, next_half_L = 0.0f, next_lo = 0.0f, next_hi = 0.0f;
+        int next_H = 0;
+        if (want_planes) {
+            next_inv = inverse_scale(__ldg(p.next_scale));
+            next_H = 1 << (p.next_bits - 1);
+            next_half_L = 0.5f * (float)((1 << p.next_bits) - 1);
+            next_lo = (float)(-next_H); next_hi = (float)next_H - 0.5f;
+        }
 #pragma unroll 1
         for (int o = 0; o < oc; ++o) {
             uint32_t acc = 0u;
@@ -184,8 +199,44 @@ window3x3c64_kernel(const BranchParams p) {
                 float f = __fmul_rn((float)v, alpha_s[o]);
                 if (p.residual) f = __fadd_rn(f, __ldg(p.residual + idx));
                 if (p.relu) f = fmaxf(f, 0.0f);
-                p.out_f32[idx] = f;
+                if (p.out_f32) p.out_f32[idx] = f;
                 seen_max = fmaxf(seen_max, f);
+                if (want_planes) {
+                    const int u = p.next_act == MPQ_ACT_HRELU
+                                      ? level_index<MPQ_ACT_HRELU>(f, next_inv, next_half_L, next_lo, next_hi, next_H)
+                                      : level_index<MPQ_ACT_HTANH>(f, next_inv, next_half_L, next_lo, next_hi, next_H);
+                    code_s[o * 256 + tid] = (unsigned char)u;
+                }
+            }
+        }
+        if (want_planes) {
+            // the pixel's level indices, 32 channels at a time, through the 8 x 8 bit-block transpose:
+            // word i of a group holds channels i, 8 + i, 16 + i, 24 + i (O is a multiple of 32)
+            const int Ow = p.O / 32;
+            const int64_t plane_words_out = (int64_t)p.N * hw * Ow;
+            for (int grp = 0; grp < oc / 32; ++grp) {
+                uint32_t w8[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const unsigned char* c = code_s + (32 * grp + i) * 256 + tid;
+                    w8[i] = (uint32_t)c[0] | ((uint32_t)c[8 * 256] << 8) | ((uint32_t)c[16 * 256] << 16) | ((uint32_t)c[24 * 256] << 24);
+                }
+#pragma unroll
+                for (int d = 1; d <= 4; d *= 2) {
+                    const uint32_t mask = d == 1 ? 0x55555555u : d == 2 ? 0x33333333u : 0x0F0F0F0Fu;
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        if ((i & d) == 0) {
+                            const uint32_t x = ((w8[i] >> d) ^ w8[i + d]) & mask;
+                            w8[i + d] ^= x;
+                            w8[i] ^= x << d;
+                        }
+                    }
+                }
+                const int64_t at0 = ((int64_t)n * hw + rem) * Ow + (o_base / 32 + grp);
+#pragma unroll
+                for (int q = 0; q < 8; ++q)
+                    if (q < p.next_bits) p.next_planes[(int64_t)q * plane_words_out + at0] = w8[q];
             }
         }
     }
@@ -198,8 +249,7 @@ window3x3c64_kernel(const BranchParams p) {
 
 // (activations of up to 4 bits: 18 words per plane must stay in registers)
 inline bool window3x3c64_applies(const BranchParams& p, int a_bits) {
-    return p.KH == 3 && p.KW == 3 && p.Cw == 2 && a_bits <= 4 && p.next_planes == nullptr &&
-           (p.pad == 0 || p.tap_sums != nullptr);
+    return p.KH == 3 && p.KW == 3 && p.Cw == 2 && a_bits <= 4 && (p.pad == 0 || p.tap_sums != nullptr);
 }
 
 template <int HB, int SB>
@@ -215,7 +265,14 @@ static int launch_window3x3c64(const BranchParams& p, cudaStream_t st) {
     attr[0].val.programmaticStreamSerializationAllowed = bx * by >= 1024 ? 1 : 0;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    if (cudaLaunchKernelEx(&cfg, window3x3c64_kernel<HB, SB>, p) != cudaSuccess) {
+    // weights, decoder factors, tap sums, level-index tile
+    constexpr size_t smem_bytes = (size_t)kWindowChannels * (HB * 5 * sizeof(uint4) + sizeof(float) + 9 * sizeof(int) + 256);
+    static PerDeviceOnce configured[2];
+    const bool planes = p.next_planes != nullptr;
+    auto kern = planes ? window3x3c64_kernel<HB, SB, true> : window3x3c64_kernel<HB, SB, false>;
+    if (configured[planes ? 1 : 0].raise_smem_limit(kern, smem_bytes) != MPQ_OK) return MPQ_ERR_CUDA;
+    cfg.dynamicSmemBytes = smem_bytes;
+    if (cudaLaunchKernelEx(&cfg, kern, p) != cudaSuccess) {
         cudaGetLastError();
         return MPQ_ERR_CUDA;
     }
